@@ -1,0 +1,136 @@
+"""Layer tables of the synthetic workloads and the per-layer cost model (MACs, compulsory bytes).
+
+Shapes follow the networks the paper measures (WideResNet-40-2 on 32x32 images, ResNet-34 on
+224x224 images, Section IV-A) with every 3x3 convolution read as a grouped 3x3 convolution, plus a
+ResNeXt-50-32x4d-shaped family and a group-count sweep down to depthwise.  The MAC count is
+Eq. (2) of the paper.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import List
+
+
+@dataclass(frozen=True)
+class Layer:
+    name: str
+    N: int
+    C_in: int
+    H: int
+    W: int
+    C_out: int
+    KH: int = 3
+    KW: int = 3
+    stride: int = 1
+    pad: int = 1
+    dilation: int = 1
+    groups: int = 1
+    x_dist: str = "uniform"
+    repeat: int = 1  # how many times the layer occurs in its stack
+
+    @property
+    def Cg(self) -> int:
+        return self.C_in // self.groups
+
+    @property
+    def Kg(self) -> int:
+        return self.C_out // self.groups
+
+    @property
+    def H_out(self) -> int:
+        return (self.H + 2 * self.pad - self.dilation * (self.KH - 1) - 1) // self.stride + 1
+
+    @property
+    def W_out(self) -> int:
+        return (self.W + 2 * self.pad - self.dilation * (self.KW - 1) - 1) // self.stride + 1
+
+    @property
+    def macs(self) -> int:
+        """Eq. (2): N*C_in*C_out*KH*KW*H_out*W_out / g."""
+        return self.N * self.C_in * self.C_out * self.KH * self.KW * self.H_out * self.W_out // self.groups
+
+    @property
+    def flops(self) -> int:
+        return 2 * self.macs
+
+    @property
+    def x_elems(self) -> int:
+        return self.N * self.C_in * self.H * self.W
+
+    @property
+    def y_elems(self) -> int:
+        return self.N * self.C_out * self.H_out * self.W_out
+
+    @property
+    def w_elems(self) -> int:
+        return self.C_out * self.Cg * self.KH * self.KW
+
+    @property
+    def compulsory_bytes(self) -> int:
+        """x read once + y written once + w read once, fp32."""
+        return 4 * (self.x_elems + self.y_elems + self.w_elems)
+
+    def desc_args(self):
+        return (self.N, self.C_in, self.H, self.W, self.C_out, self.KH, self.KW, self.stride, self.pad,
+                self.dilation, self.groups)
+
+    def with_(self, **kw) -> "Layer":
+        return replace(self, **kw)
+
+
+def config0() -> List[Layer]:
+    """Single small layer: 64->64 @16x16, 3x3, groups 4, N=1."""
+    return [Layer("cfg0_64x16_g4", 1, 64, 16, 16, 64, groups=4)]
+
+
+def wrn_stack(groups: int, N: int) -> List[Layer]:
+    """WideResNet-40-2-shaped stack: channels 32/64/128 at 32/16/8, six 3x3 layers per stage, the
+    first layer of stages 2 and 3 has stride 2 and widens the channel count."""
+    g = groups
+    return [
+        Layer("wrn_s1_32@32", N, 32, 32, 32, 32, groups=g, repeat=6),
+        Layer("wrn_s2t_32-64@32s2", N, 32, 32, 32, 64, stride=2, groups=g, repeat=1),
+        Layer("wrn_s2_64@16", N, 64, 16, 16, 64, groups=g, repeat=5),
+        Layer("wrn_s3t_64-128@16s2", N, 64, 16, 16, 128, stride=2, groups=g, repeat=1),
+        Layer("wrn_s3_128@8", N, 128, 8, 8, 128, groups=g, repeat=5),
+    ]
+
+
+WRN_GROUPS = (1, 2, 4, 8, 16)
+WRN_BATCHES = (1, 128)
+
+
+def resnet34_layers(groups: int, N: int) -> List[Layer]:
+    """ResNet-34-shaped 3x3 layers at 224x224 input: 64/128/256/512 channels at 56/28/14/7."""
+    g = groups
+    return [
+        Layer("r34_64@56", N, 64, 56, 56, 64, groups=g),
+        Layer("r34_64-128@56s2", N, 64, 56, 56, 128, stride=2, groups=g),
+        Layer("r34_128@28", N, 128, 28, 28, 128, groups=g),
+        Layer("r34_128-256@28s2", N, 128, 28, 28, 256, stride=2, groups=g),
+        Layer("r34_256@14", N, 256, 14, 14, 256, groups=g),
+        Layer("r34_256-512@14s2", N, 256, 14, 14, 512, stride=2, groups=g),
+        Layer("r34_512@7", N, 512, 7, 7, 512, groups=g),
+    ]
+
+
+R34_GROUPS = (1, 2, 4, 8, 16, 32)
+R34_BATCHES = (1, 64)
+
+
+def resnext_layers(N: int = 64) -> List[Layer]:
+    """ResNeXt-50-32x4d-shaped bottleneck middle convs: 3x3, 32 groups, N(0,1) inputs."""
+    mk = lambda name, C, HW, s: Layer(name, N, C, HW, HW, C, stride=s, groups=32, x_dist="normal")
+    return [
+        mk("rx_128@56", 128, 56, 1), mk("rx_256@56s2", 256, 56, 2), mk("rx_256@28", 256, 28, 1),
+        mk("rx_512@28s2", 512, 28, 2), mk("rx_512@14", 512, 14, 1), mk("rx_1024@14s2", 1024, 14, 2),
+        mk("rx_1024@7", 1024, 7, 1),
+    ]
+
+
+SWEEP_GROUPS = (1, 2, 4, 8, 16, 32, 64, 128, 256)
+
+
+def sweep_layers(N: int = 32) -> List[Layer]:
+    """Group-count sweep to depthwise: 256->256 @56x56, 3x3, stride 1, pad 1."""
+    return [Layer("sweep_256@56_g%d" % g, N, 256, 56, 56, 256, groups=g) for g in SWEEP_GROUPS]
