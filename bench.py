@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of libgconv on B200: grouped-conv GFLOP/s and ms/layer vs groups, % of roofline.
+
+One "step" = one pass of the hot path over the WideResNet-40-2-shaped stack (18 grouped 3x3
+layers: 32/64/128 channels at 32/16/8, stride-2 transitions) at batch 128 for every group count in
+{1,2,4,8,16}: 90 gconv_forward launches.  Every layer instance owns its x and y buffers, so ~1.8 GB
+is cycled between two uses of the same buffer (more than the 126 MB L2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is GFLOP/s (2*MACs of Eq. (2) of the paper per second) with inputs
+resident in HBM, the step replayed as a CUDA graph; `e2e` is the same metric through
+gconv_forward_host with pinned host buffers (copies inside the timed region).  `--impl reference`
+times the CPU oracle (the only reference there is: the paper ships no code) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2006_09791_b200 import synth, workloads as wl  # noqa: E402
+
+METRIC = "grouped_conv_gflops"
+UNIT = "GFLOP/s"
+WORKLOAD = "wrn40_2_stack_N128_groups_1_2_4_8_16"
+BATCH = 128
+CPU_SAMPLE_BATCH = 8
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def step_layers(batch):
+    """[(groups, Layer)] of one step, repeats expanded (90 entries at the full workload)."""
+    out = []
+    for g in wl.WRN_GROUPS:
+        for L in wl.wrn_stack(g, batch):
+            out.extend([(g, L)] * L.repeat)
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm
+def oracle_sample_time(batch, threads):
+    """Runs the oracle as it stands over the stack at a reduced batch; returns (seconds, macs)."""
+    import oracle
+    total_macs, total_s = 0, 0.0
+    cache = {}
+    for g in wl.WRN_GROUPS:
+        for L in wl.wrn_stack(g, batch):
+            key = (L.C_in, L.H, L.C_out, g)
+            if key not in cache:
+                cache[key] = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, g, synth.layer_seed(1, *key))
+            x, w = cache[key]
+            t0 = time.perf_counter()
+            for _ in range(L.repeat):
+                oracle.gconv_ref(x, w, L.stride, L.pad, L.dilation, g, threads=threads)
+            total_s += time.perf_counter() - t0
+            total_macs += L.macs * L.repeat
+    return total_s, total_macs
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    sample = "the 18-layer stack at N=%d (of %d) for every group count, oracle as it stands" % (CPU_SAMPLE_BATCH, BATCH)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_time(1, threads)
+    secs, macs = 0.0, 0
+    for _ in range(args.steps):
+        s, m = oracle_sample_time(CPU_SAMPLE_BATCH, threads)
+        secs += s
+        macs += m
+    value = 2.0 * macs / secs / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+class Instance:
+    """One layer instance of the step: descriptor, packed weights, its own x and y buffers."""
+
+    def __init__(self, g, L, x_dev, wp, torch, gconv):
+        self.g, self.L = g, L
+        self.desc = gconv.gconv_desc_create(*L.desc_args())
+        self.x = x_dev
+        self.wp = wp
+        self.y = torch.empty(L.y_elems, dtype=torch.float32, device=x_dev.device)
+
+
+def time_layer(torch, gconv, L, stream, reps=40, min_cycle_bytes=2 * L2_BYTES + (64 << 20)):
+    """Average device time of one gconv_forward launch of layer L with cold L2: launches rotate over
+    enough distinct (x, y) buffer pairs that more than twice the L2 is cycled between reuses."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    per = 4 * (L.x_elems + L.y_elems)
+    nbuf = max(2, -(-min_cycle_bytes // per))
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.groups, 99, L.x_dist)
+        w = torch.from_numpy(w0).to(dev)
+        reps_x = -(-L.N // x0.shape[0])
+        xs = [torch.from_numpy(x0).to(dev).repeat(reps_x, 1, 1, 1)[:L.N].contiguous() for _ in range(nbuf)]
+        ys = [torch.empty(L.y_elems, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+        wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+        with torch.cuda.stream(stream):
+            gconv.gconv_pack_weights(d, w, wp, stream)
+            for i in range(min(nbuf, 5) + 3):
+                gconv.gconv_forward(d, xs[i % nbuf], wp, ys[i % nbuf], stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            graph = torch.cuda.CUDAGraph()
+            stream.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(reps):
+                    gconv.gconv_forward(d, xs[i % nbuf], wp, ys[i % nbuf], stream)
+            graph.replay()
+            stream.synchronize()
+            times = []
+            for _ in range(5):
+                e0.record(stream)
+                graph.replay()
+                e1.record(stream)
+                stream.synchronize()
+                times.append(e0.elapsed_time(e1) / reps)
+        st = gconv.gconv_last_status(d, stream)
+        assert st == 0, gconv.status_string(st)
+        return statistics.median(times), gconv.gconv_variant(d)
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def layer_row(L, ms, variant, peaks, gconv):
+    """Per-layer line of the metric: ms, GFLOP/s, achieved GB/s on compulsory bytes, % of roofline."""
+    tf32_peak = 0.5 * peaks["bf16_tflops"] * 1e12
+    fp32_peak = 148 * 128 * 2 * 1.965e9
+    pipe_peak = tf32_peak if variant == gconv.GCONV_VARIANT_IGEMM_TF32 else fp32_peak
+    t_hbm = L.compulsory_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_pipe = L.flops / pipe_peak
+    t_roof = max(t_hbm, t_pipe)
+    return {"layer": L.name, "groups": L.groups, "N": L.N, "Cg": L.Cg, "Kg": L.Kg, "variant": gconv.variant_name(variant),
+            "ms": ms, "gflops": L.flops / (ms * 1e-3) / 1e9, "gbs": L.compulsory_bytes / (ms * 1e-3) / 1e9,
+            "roofline_ms": t_roof * 1e3, "bound": "hbm" if t_hbm >= t_pipe else ("tensor" if pipe_peak == tf32_peak else "alu"),
+            "roofline_frac": t_roof / (ms * 1e-3)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2006_09791_b200 import build as gbuild
+    from paper_2006_09791_b200 import gconv
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgconv has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        gbuild.build()
+    if world > 1:
+        dist.barrier()
+    gconv.load()
+    peaks = load_peaks()
+    stream = torch.cuda.Stream(device=dev)
+
+    # ---- set up the step: every layer instance with its own buffers --------------------------------
+    plan = step_layers(BATCH)
+    host_x, host_y, dev_w = {}, {}, {}
+    insts = []
+    for g, L in plan:
+        key = (L.name, g)
+        if key not in host_x:
+            x2, w = synth.make_layer_tensors(2, L.C_in, L.H, L.W, L.C_out, 3, 3, g, synth.layer_seed(2, L.C_in, L.H, L.C_out, g))
+            hx = torch.from_numpy(x2).repeat(BATCH // 2, 1, 1, 1).contiguous().pin_memory()
+            host_x[key] = hx
+            host_y[key] = torch.empty(L.y_elems, dtype=torch.float32).pin_memory()
+            d = gconv.gconv_desc_create(*L.desc_args())
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
+            gconv.gconv_desc_destroy(d)
+            dev_w[key] = wp
+        insts.append(Instance(g, L, host_x[key].to(dev), dev_w[key], torch, gconv))
+    torch.cuda.synchronize()
+    step_macs = sum(i.L.macs for i in insts)
+    step_flops = 2 * step_macs
+    launches_per_step = sum(gconv.gconv_forward_launches(i.desc) for i in insts)
+
+    def step_device():
+        for it in insts:
+            gconv.gconv_forward(it.desc, it.x, it.wp, it.y, stream)
+
+    def step_host():
+        for it in insts:
+            key = (it.L.name, it.g)
+            gconv.gconv_forward_host(it.desc, host_x[key], it.wp, host_y[key], it.x, it.y, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing: the step as one CUDA graph ----------------------------------------
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            step_device()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step_device()
+        graph.replay()
+        stream.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record(stream)
+    barrier()
+    ms_dev = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    clocks = sampler.stop()
+    for it in insts:
+        st = gconv.gconv_last_status(it.desc, stream)
+        assert st == 0, gconv.status_string(st)
+
+    # ---- end to end through the host-buffer entry point --------------------------------------------
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            step_host()
+    e2e_steps = max(1, min(args.steps, 10))
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            step_host()
+        e1.record(stream)
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+    h2d = sum(4 * i.L.x_elems for i in insts)
+    d2h = sum(4 * i.L.y_elems for i in insts)
+
+    # ---- per-layer table (the metric proper) and roofline of the dominant kernel --------------------
+    rows, extra = [], {}
+    if rank == 0:
+        seen = {}
+        for g, L in plan:
+            key = (L.name, g)
+            if key in seen:
+                continue
+            ms, v = time_layer(torch, gconv, L, stream)
+            seen[key] = (ms, v, L)
+            rows.append(layer_row(L, ms, v, peaks, gconv))
+        by_variant = {}
+        for (name, g), (ms, v, L) in seen.items():
+            a = by_variant.setdefault(v, {"ms": 0.0, "bytes": 0, "flops": 0, "launches": 0})
+            a["ms"] += ms * L.repeat
+            a["bytes"] += L.compulsory_bytes * L.repeat
+            a["flops"] += L.flops * L.repeat
+            a["launches"] += L.repeat
+        dom_v = max(by_variant, key=lambda k: by_variant[k]["ms"])
+        dom = by_variant[dom_v]
+        t_hbm = dom["bytes"] / (peaks["hbm_gbs"] * 1e9)
+        pipe_peak = 0.5 * peaks["bf16_tflops"] * 1e12 if dom_v == gconv.GCONV_VARIANT_IGEMM_TF32 else 148 * 128 * 2 * 1.965e9
+        t_pipe = dom["flops"] / pipe_peak
+        if t_hbm >= t_pipe:
+            ach = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "traffic": None}
+        else:
+            ach = dom["flops"] / (dom["ms"] * 1e-3) / 1e12
+            roofline = {"bound": "tensor" if dom_v == gconv.GCONV_VARIANT_IGEMM_TF32 else "alu", "achieved": ach,
+                        "peak": pipe_peak / 1e12, "unit": "TFLOP/s", "frac": ach / (pipe_peak / 1e12), "traffic": None}
+        roofline.update({"kernel": gconv.variant_name(dom_v), "launches_per_step": dom["launches"],
+                         "share_of_step": dom["ms"] / sum(a["ms"] for a in by_variant.values()),
+                         "peak_source": peaks["source"]})
+        extra["roofline"] = roofline
+        # time per group count (the paper's acceptance property: time falls as g rises)
+        extra["ms_by_groups"] = {str(g): sum(ms * L.repeat for (n, gg), (ms, v, L) in seen.items() if gg == g)
+                                 for g in wl.WRN_GROUPS}
+        if args.sweep:
+            sweep_rows = []
+            for L in wl.sweep_layers(32) + wl.resnext_layers(64):
+                ms, v = time_layer(torch, gconv, L, stream, reps=20)
+                sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
+            extra["sweep_layers"] = sweep_rows
+
+    # ---- CPU baseline (rank 0, N=1 only) -----------------------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+        secs, macs = oracle_sample_time(CPU_SAMPLE_BATCH, threads)
+        cpu = {"value": 2.0 * macs / secs / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": secs,
+               "sample": "the 18-layer stack at N=%d (of %d) for every group count, oracle as it stands" % (CPU_SAMPLE_BATCH, BATCH)}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": world * step_flops / (ms_dev * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_dev, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32+tf32", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "layers_per_step": len(insts), "batch": BATCH, "groups": list(wl.WRN_GROUPS),
+                           "parallelism": "replicas only (%d)" % world, "launch": "cuda graph of the step",
+                           "l2": "every layer instance owns its x/y buffers: %.2f GB cycled per step > 126 MB L2"
+                                 % ((h2d + d2h) / 1e9)},
+                "clocks": clocks,
+                "e2e": {"value": world * step_flops / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                "gpu_launches": launches_per_step * args.steps,
+                "cpu_baseline": cpu, "layers": rows}
+        line.update(extra)
+        print(json.dumps(line))
+    for it in insts:
+        gconv.gconv_desc_destroy(it.desc)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="also time the group-count sweep and ResNeXt-shaped layers")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,161 @@
+/*
+ * libgconv -- forward grouped 2-D convolution for NVIDIA B200 (sm_100a), fp32 NCHW.
+ *
+ * The operation is the grouped convolution G(g) of Section II of the paper ("Optimizing Grouped
+ * Convolutions on Edge Devices"): C_out filters are split into g groups and each group sees only
+ * its own C_in/g input channels.  With Cg = C_in/groups (the paper's CPG), Kg = C_out/groups (the
+ * paper's KPG), in the index form of the convolution stage of Algorithm 1 (cross-correlation on
+ * the zero-padded input, no kernel flip):
+ *
+ *   y[n, g*Kg + k, p, q] = sum_{c<Cg} sum_{r<KH} sum_{s<KW}
+ *       x[n, g*Cg + c, p*stride + r*dilation - pad, q*stride + s*dilation - pad] * w[g*Kg + k, c, r, s]
+ *
+ *   H_out = floor((H + 2*pad - dilation*(KH-1) - 1)/stride) + 1, likewise W_out.
+ *
+ * Layouts (Section III-A footnote: row-major 4-D arrays):
+ *   x  [N, C_in, H, W]            fp32, device memory
+ *   w  [C_out, Cg, KH, KW]        fp32, device memory
+ *   y  [N, C_out, H_out, W_out]   fp32, device memory
+ *
+ * Conventions for every call:
+ *   - C linkage, no exceptions cross the boundary; every call that can fail returns an int status,
+ *     GCONV_OK (0) on success.
+ *   - "device" pointers are CUDA device pointers of the current device, "host" pointers are host
+ *     memory.  The caller owns every buffer and the stream; the library owns only the descriptor
+ *     and a 16-byte device status block it allocates on the first pack/forward call of a descriptor.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  pack and
+ *     forward only enqueue work on it and return without synchronising.
+ *   - Device pointers must be 16-byte aligned (GCONV_ERR_ALIGNMENT otherwise).
+ *   - There is no CPU fallback: without a CUDA device pack/forward return GCONV_ERR_CUDA.
+ */
+#ifndef GCONV_H_
+#define GCONV_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gconv_desc *gconv_desc_t; /* opaque; created/destroyed by the library */
+
+enum gconv_status {
+    GCONV_OK = 0,
+    GCONV_ERR_NULL = 1,          /* a required pointer argument is NULL */
+    GCONV_ERR_INVALID_ARG = 2,   /* a shape parameter is out of range or channels do not divide by groups */
+    GCONV_ERR_UNSUPPORTED = 3,   /* the requested kernel variant cannot run this shape */
+    GCONV_ERR_ALIGNMENT = 4,     /* a device pointer is not 16-byte aligned */
+    GCONV_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed; see gconv_last_cuda_error */
+    GCONV_ERR_PACK_MISMATCH = 6, /* device status: w_packed was packed for another shape or variant */
+    GCONV_ERR_TIMEOUT = 7        /* device status: a bounded wait inside a kernel ran out */
+};
+
+/* Kernel variants.  The numeric tolerance of a result follows the variant that produced it:
+ * max|y - y_ref| / max|y_ref| <= 1e-5 for the FP32 variants, <= 5e-3 for the TF32 variant. */
+enum gconv_variant_id {
+    GCONV_VARIANT_AUTO = 0,           /* let the selector choose (default) */
+    GCONV_VARIANT_DIRECT_GENERIC = 1, /* FP32 FFMA, one thread per output, any shape */
+    GCONV_VARIANT_DIRECT_TILED = 2,   /* FP32 FFMA, shared-memory halo + register tiles; 3x3, dilation 1, narrow groups */
+    GCONV_VARIANT_IGEMM_TF32 = 3      /* TF32 tcgen05 implicit GEMM per group; 3x3, stride 1, pad 1, Cg,Kg multiples of 8/16 */
+};
+
+/*
+ * gconv_desc_create -- describe one grouped-convolution problem (Section II; the divisibility rule
+ * "input and output channels divisible by the number of groups" is Section III-B).
+ *   out       host pointer receiving the handle (library-owned until gconv_desc_destroy).
+ *   N..groups problem sizes; stride, pad and dilation apply to both spatial axes.
+ * Host only: touches no device, so it works without a GPU.  Picks the kernel variant with the
+ * built-in selector (keyed on Cg, Kg, H*W, N; see gconv_variant).
+ * Errors: GCONV_ERR_NULL (out), GCONV_ERR_INVALID_ARG (any size < 1, stride < 1, dilation < 1,
+ * pad < 0, C_in or C_out not divisible by groups, empty output, or a tensor over 2^40 elements).
+ */
+int gconv_desc_create(gconv_desc_t *out, int N, int C_in, int H, int W, int C_out, int KH, int KW,
+                      int stride, int pad, int dilation, int groups);
+
+/* Frees the descriptor and its device status block.  NULL is accepted. */
+int gconv_desc_destroy(gconv_desc_t desc);
+
+/* Output spatial size from the floor formula above.  Host only. */
+int gconv_out_shape(gconv_desc_t desc, int *H_out, int *W_out);
+
+/* Multiply-accumulate count of the layer, Eq. (2) of the paper:
+ * N*C_in*C_out*KH*KW*H_out*W_out/groups.  Returns -1 for a NULL descriptor. */
+long long gconv_macs(gconv_desc_t desc);
+
+/* Size in bytes of the packed-weight buffer for the descriptor's current variant (0 for NULL). */
+size_t gconv_packed_bytes(gconv_desc_t desc);
+
+/* The variant the descriptor will run (never GCONV_VARIANT_AUTO), or -1 for NULL. */
+int gconv_variant(gconv_desc_t desc);
+
+/* 1 if `variant` can run this shape, else 0. */
+int gconv_variant_supported(gconv_desc_t desc, int variant);
+
+/*
+ * Force a variant (tests, selector training) or return to the selector's choice with
+ * GCONV_VARIANT_AUTO.  Packed weights are variant-specific: call before gconv_pack_weights and
+ * re-pack after changing it.  Errors: GCONV_ERR_NULL, GCONV_ERR_INVALID_ARG (unknown id),
+ * GCONV_ERR_UNSUPPORTED (the variant cannot run this shape; the descriptor is left unchanged).
+ */
+int gconv_desc_set_variant(gconv_desc_t desc, int variant);
+
+/*
+ * gconv_pack_weights -- the kernel-reshaping stage (first stage of Algorithm 1, Section III-B:
+ * it does not depend on the input, so it is done once ahead of time).  Reorders (and, for the TF32
+ * variant, rounds to TF32 with round-to-nearest) w[C_out, Cg, KH, KW] into the layout the
+ * descriptor's variant reads, prefixed by a 64-byte header that names shape and variant.
+ *   w_ochw    device, fp32 [C_out, Cg, KH, KW], read only.
+ *   w_packed  device, gconv_packed_bytes(desc) bytes, written.  The blob is position independent
+ *             and may be copied, saved and reloaded.
+ * One kernel launch on `stream`.  Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_CUDA.
+ */
+int gconv_pack_weights(gconv_desc_t desc, const float *w_ochw, void *w_packed, void *stream);
+
+/*
+ * gconv_forward -- the grouped convolution itself (Section II; Algorithm 1's input-reshaping,
+ * convolution and output-reshaping stages fused into one kernel: the input tile is staged in
+ * shared memory and y is written directly in NCHW).
+ *   x_nchw    device, fp32 [N, C_in, H, W], read only; must not overlap y.
+ *   w_packed  device, produced by gconv_pack_weights on a descriptor of the same shape and variant.
+ *   y_nchw    device, fp32 [N, C_out, H_out, W_out], every element written.
+ * Kernel launches only, on `stream`; deterministic (no atomics on y).  A w_packed made for another shape or
+ * variant is detected on the device: y is left unwritten and gconv_last_status reports
+ * GCONV_ERR_PACK_MISMATCH.  Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_CUDA.
+ */
+int gconv_forward(gconv_desc_t desc, const float *x_nchw, const void *w_packed, float *y_nchw, void *stream);
+
+/*
+ * gconv_forward_host -- the same operation for callers whose activations live in host memory:
+ * copies x to the device, runs gconv_forward and copies y back, all enqueued on `stream` in order.
+ *   x_host    host, fp32 [N, C_in, H, W] (pinned memory makes the copies asynchronous).
+ *   y_host    host, fp32 [N, C_out, H_out, W_out], written when the stream reaches that point.
+ *   x_stage, y_stage   device staging buffers of the sizes of x and y, caller-owned.
+ *   w_packed  device, as for gconv_forward.
+ * Errors as gconv_forward.
+ */
+int gconv_forward_host(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host,
+                       float *x_stage, float *y_stage, void *stream);
+
+/* Number of kernel launches one gconv_forward of this descriptor enqueues (for launch accounting). */
+int gconv_forward_launches(gconv_desc_t desc);
+
+/*
+ * Synchronises `stream`, then reads and clears the descriptor's device status word: GCONV_OK, or
+ * the first of GCONV_ERR_PACK_MISMATCH / GCONV_ERR_TIMEOUT a kernel of this descriptor recorded.
+ * A kernel that records an error returns early; it never traps.  GCONV_ERR_CUDA if the sync fails.
+ */
+int gconv_last_status(gconv_desc_t desc, void *stream);
+
+/* The cudaError_t (as int) of the last failed CUDA call made for this descriptor, 0 if none. */
+int gconv_last_cuda_error(gconv_desc_t desc);
+
+/* Static, NUL-terminated description of a status code. */
+const char *gconv_status_string(int status);
+
+/* Static name of a variant id ("direct_generic", ...), or "unknown". */
+const char *gconv_variant_name(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GCONV_H_ */

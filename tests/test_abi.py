@@ -1,0 +1,78 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates descriptors and reports shapes/MACs."""
+import os
+import re
+
+import pytest
+
+from paper_2006_09791_b200 import build as gbuild
+from paper_2006_09791_b200 import gconv
+from paper_2006_09791_b200.workloads import Layer, config0, resnet34_layers, wrn_stack
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gbuild.build()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "gconv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gconv_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_exports_every_declared_symbol():
+    lib = gconv.load()
+    names = _declared_symbols()
+    assert "gconv_desc_create" in names and "gconv_pack_weights" in names and "gconv_forward" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(gconv._SIGNATURES), set(names) ^ set(gconv._SIGNATURES)
+
+
+def test_descriptor_queries():
+    for L in config0() + wrn_stack(4, 128) + resnet34_layers(32, 64):
+        d = gconv.gconv_desc_create(*L.desc_args())
+        try:
+            assert gconv.gconv_out_shape(d) == (L.H_out, L.W_out)
+            assert gconv.gconv_macs(d) == L.macs
+            v = gconv.gconv_variant(d)
+            assert v in gconv.VARIANT_TOLERANCE and gconv.gconv_variant_supported(d, v)
+            assert gconv.gconv_packed_bytes(d) >= 4 * L.w_elems
+            assert gconv.gconv_forward_launches(d) >= 1
+        finally:
+            gconv.gconv_desc_destroy(d)
+
+
+@pytest.mark.parametrize("args", [
+    (0, 8, 8, 8, 8, 3, 3, 1, 1, 1, 1), (1, 6, 8, 8, 8, 3, 3, 1, 1, 1, 4), (1, 8, 8, 8, 6, 3, 3, 1, 1, 1, 4),
+    (1, 8, 8, 8, 8, 3, 3, 0, 1, 1, 1), (1, 8, 8, 8, 8, 3, 3, 1, -1, 1, 1), (1, 8, 8, 8, 8, 3, 3, 1, 1, 0, 1),
+    (1, 8, 2, 2, 8, 5, 5, 1, 0, 1, 1), (1, 8, 8, 8, 8, 3, 3, 1, 1, 1, 0), (1, 8, 4, 4, 8, 3, 3, 1, 0, 2, 1)])
+def test_rejects_invalid_descriptors(args):
+    with pytest.raises(gconv.GconvError) as e:
+        gconv.gconv_desc_create(*args)
+    assert e.value.status == gconv.GCONV_ERR_INVALID_ARG
+
+
+def test_null_and_variant_errors():
+    lib = gconv.load()
+    assert lib.gconv_desc_create(None, 1, 8, 8, 8, 8, 3, 3, 1, 1, 1, 1) == gconv.GCONV_ERR_NULL
+    assert lib.gconv_desc_destroy(None) == gconv.GCONV_OK
+    assert lib.gconv_packed_bytes(None) == 0 and lib.gconv_variant(None) == -1 and lib.gconv_macs(None) == -1
+    d = gconv.gconv_desc_create(1, 8, 8, 8, 8, 5, 5, 1, 2, 1, 2)
+    try:
+        assert lib.gconv_pack_weights(d, None, None, None) == gconv.GCONV_ERR_NULL
+        assert lib.gconv_forward(d, None, None, None, None) == gconv.GCONV_ERR_NULL
+        assert lib.gconv_pack_weights(d, 4, 16, None) == gconv.GCONV_ERR_ALIGNMENT
+        assert lib.gconv_forward(d, 16, 16, 8, None) == gconv.GCONV_ERR_ALIGNMENT
+        assert lib.gconv_desc_set_variant(d, 99) == gconv.GCONV_ERR_INVALID_ARG
+        # a 5x5 kernel is outside what the tiled and tensor-core variants accept
+        assert lib.gconv_desc_set_variant(d, gconv.GCONV_VARIANT_IGEMM_TF32) == gconv.GCONV_ERR_UNSUPPORTED
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_DIRECT_GENERIC
+        gconv.gconv_desc_set_variant(d, gconv.GCONV_VARIANT_DIRECT_GENERIC)
+        gconv.gconv_desc_set_variant(d, gconv.GCONV_VARIANT_AUTO)
+    finally:
+        gconv.gconv_desc_destroy(d)
+    assert gconv.status_string(gconv.GCONV_ERR_TIMEOUT) and gconv.variant_name(3) == "igemm_tf32"

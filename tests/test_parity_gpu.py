@@ -1,0 +1,145 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
+inputs, element by element over the whole tensor.  Bar: max|y-y_ref|/max|y_ref| <= 1e-5 for the
+FP32 variants and <= 5e-3 for the TF32 variant."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2006_09791_b200 import build as gbuild
+from paper_2006_09791_b200 import gconv, synth
+from paper_2006_09791_b200.workloads import Layer, config0, resnet34_layers, resnext_layers, sweep_layers, wrn_stack
+
+from golden_io import load_case
+from gpu_util import check_layer, rel_err, run_layer
+
+pytestmark = pytest.mark.gpu
+
+ALL_VARIANTS = [gconv.GCONV_VARIANT_DIRECT_GENERIC, gconv.GCONV_VARIANT_DIRECT_TILED, gconv.GCONV_VARIANT_IGEMM_TF32]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gbuild.build()
+
+
+def _supported(L, v):
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        return gconv.gconv_variant_supported(d, v)
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+@pytest.mark.parametrize("name", ["fig3_shape_index_valued.txt", "delta_no_flip.txt", "ones_zero_padding.txt",
+                                  "stride2_pad1.txt", "dilation2.txt", "two_groups_asymmetric.txt"])
+def test_hand_worked_cases_on_gpu(name):
+    x, w, p, y_want = load_case(name)
+    N, C_in, H, W = x.shape
+    C_out, _, KH, KW = w.shape
+    L = Layer(name, N, C_in, H, W, C_out, KH, KW, p["stride"], p["pad"], p["dilation"], p["groups"])
+    for v in ALL_VARIANTS:
+        if _supported(L, v):
+            y, _ = run_layer(L, x, w, v)
+            np.testing.assert_allclose(y, y_want, rtol=1e-6, atol=0)
+
+
+def test_config0_every_variant():
+    (L,) = config0()
+    ran = 0
+    for v in ALL_VARIANTS:
+        if _supported(L, v):
+            check_layer(L, v)
+            ran += 1
+    assert ran >= 1
+    check_layer(L)
+
+
+ODD_SHAPES = [
+    # N, C_in, H, W, C_out, KH, KW, stride, pad, dil, groups
+    (2, 6, 13, 11, 9, 3, 3, 1, 1, 1, 3), (1, 8, 17, 19, 8, 3, 3, 2, 1, 1, 8), (3, 4, 9, 33, 12, 3, 3, 1, 1, 1, 2),
+    (1, 10, 7, 7, 10, 3, 3, 1, 1, 1, 10), (2, 12, 21, 5, 6, 5, 3, 2, 2, 1, 3), (1, 16, 12, 12, 32, 1, 1, 1, 0, 1, 4),
+    (1, 6, 15, 15, 6, 3, 3, 1, 2, 2, 2), (2, 32, 16, 16, 32, 3, 3, 1, 1, 1, 2), (1, 48, 20, 24, 96, 3, 3, 1, 1, 1, 3),
+    (2, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1), (1, 32, 7, 7, 32, 3, 3, 1, 1, 1, 1), (1, 24, 56, 56, 24, 3, 3, 2, 1, 1, 24),
+    (5, 3, 37, 41, 3, 3, 3, 1, 1, 1, 3), (1, 4, 64, 130, 4, 3, 3, 1, 1, 1, 4), (2, 16, 33, 35, 16, 3, 3, 2, 1, 1, 4),
+    (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
+]
+
+
+@pytest.mark.parametrize("cfg", ODD_SHAPES)
+def test_odd_shapes_every_variant(cfg):
+    L = Layer("odd", *cfg)
+    for v in [gconv.GCONV_VARIANT_AUTO] + ALL_VARIANTS:
+        if v == gconv.GCONV_VARIANT_AUTO or _supported(L, v):
+            check_layer(L, v, seed=7)
+
+
+@pytest.mark.parametrize("groups", [1, 2, 4, 8, 16])
+def test_wrn_stack_small_batch(groups):
+    """Every distinct layer of the WRN-40-2-shaped stack at N = 1 and a ragged N = 3, all variants."""
+    for N in (1, 3):
+        for L in wrn_stack(groups, N):
+            check_layer(L)
+            for v in ALL_VARIANTS[1:]:
+                if _supported(L, v):
+                    check_layer(L, v)
+
+
+@pytest.mark.parametrize("groups", [1, 4, 32])
+def test_resnet34_shapes(groups):
+    for L in resnet34_layers(groups, 2):
+        check_layer(L)
+
+
+def test_resnext_shapes():
+    for L in resnext_layers(N=1):
+        check_layer(L)
+
+
+def test_sweep_to_depthwise_small_batch():
+    for L in sweep_layers(N=1):
+        check_layer(L)
+
+
+def test_pack_mismatch_is_reported_not_fatal():
+    (L,) = config0()
+    x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 5)
+    dev = torch.device("cuda:0")
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        wp = torch.zeros(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)  # never packed
+        y = torch.full((L.y_elems,), 7.0, dtype=torch.float32, device=dev)
+        gconv.gconv_forward(d, torch.from_numpy(x).to(dev), wp, y)
+        assert gconv.gconv_last_status(d) == gconv.GCONV_ERR_PACK_MISMATCH
+        assert bool((y == 7.0).all())
+        assert gconv.gconv_last_status(d) == gconv.GCONV_OK  # reading clears it
+        gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
+        gconv.gconv_forward(d, torch.from_numpy(x).to(dev), wp, y)
+        assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+        y_ref = oracle.gconv_ref(x, w, 1, 1, 1, L.groups)
+        assert rel_err(y.cpu().numpy().reshape(y_ref.shape), y_ref) <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(d)]
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def test_forward_host_and_second_stream():
+    L = Layer("host", 2, 16, 20, 20, 16, groups=4)
+    x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 9)
+    dev = torch.device("cuda:0")
+    s = torch.cuda.Stream()
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        with torch.cuda.stream(s):
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            w_d = torch.from_numpy(w).to(dev)
+            xs = torch.empty(L.x_elems, dtype=torch.float32, device=dev)
+            ys = torch.empty(L.y_elems, dtype=torch.float32, device=dev)
+        xh = torch.from_numpy(x).pin_memory()
+        yh = torch.empty(L.y_elems, dtype=torch.float32).pin_memory()
+        gconv.gconv_pack_weights(d, w_d, wp, s)
+        gconv.gconv_forward_host(d, xh, wp, yh, xs, ys, s)
+        assert gconv.gconv_last_status(d, s) == gconv.GCONV_OK
+        y_ref = oracle.gconv_ref(x, w, 1, 1, 1, L.groups)
+        assert rel_err(yh.numpy().reshape(y_ref.shape), y_ref) <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(d)]
+    finally:
+        gconv.gconv_desc_destroy(d)
