@@ -21,6 +21,8 @@ bool variant_supported(const Shape& s, int v) {
     switch (v) {
         case GCONV_VARIANT_DIRECT_GENERIC:
             return true;
+        case GCONV_VARIANT_DIRECT_TILED:
+            return tiled_supported(s);
         default:
             return false;
     }
@@ -29,7 +31,7 @@ bool variant_supported(const Shape& s, int v) {
 // Variant selector.  Keyed on (Cg, Kg, H*W, N) like the tile-size choice the paper leaves to
 // autotuning (Section III-C); the thresholds come from measured timings of the forced variants.
 int select_variant(const Shape& s) {
-    (void)s;
+    if (tiled_supported(s)) return GCONV_VARIANT_DIRECT_TILED;
     return GCONV_VARIANT_DIRECT_GENERIC;
 }
 
@@ -121,6 +123,8 @@ long long gconv_macs(gconv_desc_t d) {
 size_t gconv_packed_bytes(gconv_desc_t d) {
     if (d == nullptr) return 0;
     switch (d->variant) {
+        case GCONV_VARIANT_DIRECT_TILED:
+            return tiled_packed_bytes(d->s);
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             return generic_packed_bytes(d->s);
@@ -156,6 +160,9 @@ int gconv_pack_weights(gconv_desc_t d, const float* w_ochw, void* w_packed, void
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e;
     switch (d->variant) {
+        case GCONV_VARIANT_DIRECT_TILED:
+            e = tiled_pack(d->s, w_ochw, w_packed, st);
+            break;
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             e = generic_pack(d->s, w_ochw, w_packed, st);
@@ -172,6 +179,9 @@ int gconv_forward(gconv_desc_t d, const float* x, const void* w_packed, float* y
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e;
     switch (d->variant) {
+        case GCONV_VARIANT_DIRECT_TILED:
+            e = tiled_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
+            break;
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             e = generic_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);

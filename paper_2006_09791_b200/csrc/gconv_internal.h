@@ -43,4 +43,40 @@ cudaError_t generic_pack(const Shape& s, const float* w, void* packed, cudaStrea
 cudaError_t generic_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status,
                             int sm_count, cudaStream_t st);
 
+// Division by a run-time constant as multiply-high + shift; exact for numerators below 2^31.
+struct FastDiv {
+    uint32_t mul, shr, div;
+    __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const {
+        const uint32_t qq = (div != 1) ? (__umulhi(n, mul) >> shr) : n;
+        r = n - qq * div;
+        q = qq;
+    }
+};
+FastDiv make_fastdiv(uint32_t d);
+
+// DIRECT_TILED, narrow groups (Kg in {1,2,4,8}): one thread per (image, group, row strip, 4-pixel chunk).
+struct RowsCfg {
+    FastDiv div_xq, div_yt, div_g;
+    uint32_t items;
+    int PR, vec, pad01;
+};
+bool rows_supported(const Shape& s);
+RowsCfg rows_config(const Shape& s);
+cudaError_t rows_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, cudaStream_t st);
+
+// DIRECT_TILED: launch geometry chosen on the host from the shape.
+struct TiledCfg {
+    int TXT, TY, KQ, GB, KT, CCH;          // x threads, rows, filter slabs, groups per CTA, filters per thread, channel chunk
+    int IH, IW, IWP, LPR;                  // staged patch rows, columns, padded row pitch, lanes per staged row
+    int tiles_x, tiles_y, kblocks, gblocks;
+    int threads;
+    size_t smem;
+};
+bool tiled_supported(const Shape& s);
+size_t tiled_packed_bytes(const Shape& s);
+TiledCfg tiled_config(const Shape& s, int sm_count);
+cudaError_t tiled_pack(const Shape& s, const float* w, void* packed, cudaStream_t st);
+cudaError_t tiled_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
+                          cudaStream_t st);
+
 }  // namespace gconv
