@@ -23,6 +23,8 @@ bool variant_supported(const Shape& s, int v) {
             return true;
         case GCONV_VARIANT_DIRECT_TILED:
             return tiled_supported(s);
+        case GCONV_VARIANT_IGEMM_TF32:
+            return igemm_supported(s);
         default:
             return false;
     }
@@ -31,6 +33,7 @@ bool variant_supported(const Shape& s, int v) {
 // Variant selector.  Keyed on (Cg, Kg, H*W, N) like the tile-size choice the paper leaves to
 // autotuning (Section III-C); the thresholds come from measured timings of the forced variants.
 int select_variant(const Shape& s) {
+    if (igemm_supported(s) && s.Cg >= 8 && s.Kg >= 8) return GCONV_VARIANT_IGEMM_TF32;
     if (tiled_supported(s)) return GCONV_VARIANT_DIRECT_TILED;
     return GCONV_VARIANT_DIRECT_GENERIC;
 }
@@ -125,6 +128,8 @@ size_t gconv_packed_bytes(gconv_desc_t d) {
     switch (d->variant) {
         case GCONV_VARIANT_DIRECT_TILED:
             return tiled_packed_bytes(d->s);
+        case GCONV_VARIANT_IGEMM_TF32:
+            return igemm_packed_bytes(d->s);
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             return generic_packed_bytes(d->s);
@@ -163,6 +168,9 @@ int gconv_pack_weights(gconv_desc_t d, const float* w_ochw, void* w_packed, void
         case GCONV_VARIANT_DIRECT_TILED:
             e = tiled_pack(d->s, w_ochw, w_packed, st);
             break;
+        case GCONV_VARIANT_IGEMM_TF32:
+            e = igemm_pack(d->s, w_ochw, w_packed, st);
+            break;
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             e = generic_pack(d->s, w_ochw, w_packed, st);
@@ -181,6 +189,9 @@ int gconv_forward(gconv_desc_t d, const float* x, const void* w_packed, float* y
     switch (d->variant) {
         case GCONV_VARIANT_DIRECT_TILED:
             e = tiled_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
+            break;
+        case GCONV_VARIANT_IGEMM_TF32:
+            e = igemm_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
             break;
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:

@@ -79,4 +79,22 @@ cudaError_t tiled_pack(const Shape& s, const float* w, void* packed, cudaStream_
 cudaError_t tiled_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
                           cudaStream_t st);
 
+// IGEMM_TF32: tile geometry of the tcgen05 implicit-GEMM kernel.
+struct IgemmCfg {
+    int CK, chunks;          // channels per pipeline stage, stages per vertical tap
+    int Kt, NT, Np;          // filters per tile, filter tiles per group, MMA N (3*Kt padded to 16)
+    int seg_mode;            // 1: a tile is any four 32-pixel segments (W divides 32); 0: a tile is R whole rows
+    int SPI, R, RB, MT;      // segments per image; rows per tile, row blocks per image; pixel tiles in total
+    int need_xchg;           // rows may straddle a warp boundary in the epilogue
+    int num_tiles, stages, grid;
+    uint32_t stage_bytes;
+    size_t smem_bytes;
+};
+bool igemm_supported(const Shape& s);
+IgemmCfg igemm_config(const Shape& s, int sm_count);
+size_t igemm_packed_bytes(const Shape& s);
+cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_t st);
+cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
+                          cudaStream_t st);
+
 }  // namespace gconv
