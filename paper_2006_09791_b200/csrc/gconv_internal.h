@@ -85,6 +85,7 @@ struct IgemmCfg {
     int Kt, NT, Np;          // filters per tile, filter tiles per group, MMA N (3*Kt padded to 16)
     int seg_mode;            // 1: a tile is any four 32-pixel segments (W divides 32); 0: a tile is R whole rows
     int SPI, R, RB, MT;      // segments per image; rows per tile, row blocks per image; pixel tiles in total
+    int seg_fstep;           // flat-pixel step between consecutive segments of an image
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int num_tiles, stages, grid;
     uint32_t stage_bytes;

@@ -21,6 +21,8 @@
 //   * D lives in TMEM (3*Kt <= 192 fp32 columns, double buffered), the epilogue warps read it with
 //     tcgen05.ld, apply the horizontal shifts with warp shuffles and write y directly in NCHW with
 //     128-byte coalesced rows.
+// Stride 2 (pad 1) keeps the even rows and columns of that stride-1 result: same operands, the
+// epilogue stores only those lanes (and for W = 32 the odd rows are never loaded or multiplied).
 // All groups and all images run in one persistent launch: the tile index enumerates
 // (group, filter tile, pixel tile), one CTA per SM walks it.
 //
@@ -180,6 +182,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
     const uint32_t a_bytes = 4u * (uint32_t)c.CK * 128u;
     const uint32_t b_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;
     const int HW = s.H * s.W;
+    const size_t OHW = (size_t)s.H_out * s.W_out;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -197,7 +200,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                     if (c.seg_mode) {
                         const int sg = mt * 4 + j;
                         int n = sg / c.SPI;
-                        seg_f[j] = (sg - n * c.SPI) * 32;
+                        seg_f[j] = (sg - n * c.SPI) * c.seg_fstep;
                         seg_n[j] = n < s.N ? n : s.N;   // past the last image: fully out of bounds, zero fill
                     } else {
                         const int n = mt / c.RB;
@@ -279,21 +282,27 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             if (c.seg_mode) {
                 const int sg = mt * 4 + wq;
                 n = sg / c.SPI;
-                f = (sg - n * c.SPI) * 32 + lane;
+                f = (sg - n * c.SPI) * c.seg_fstep + lane;
                 valid = n < s.N;
             } else {
                 n = mt / c.RB;
                 f = (mt - n * c.RB) * c.R * s.W + l;
                 valid = (l < c.R * s.W) && (f < HW);
             }
-            const int q = f % s.W;
+            const int prow = f / s.W;
+            const int q = f - prow * s.W;
             const bool use_left = q > 0;
             const bool use_right = q < s.W - 1;
+            int fo = f;                                  // position in the output plane
+            if (s.stride == 2) {                         // stride 2 keeps the even rows and columns of the stride-1 result
+                valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
+                fo = (prow >> 1) * s.W_out + (q >> 1);
+            }
             const uint32_t buf = tcount & 1;
             if (!mbar_wait(smem_u32(&ctl.tmem_full[buf]), (tcount >> 1) & 1, abort_flag, status, 400 + buf)) break;
             tc_fence_after();
             const uint32_t t0 = tmem_base + buf * kAccStride + ((uint32_t)(wq * 32) << 16);
-            float* yk = y + ((size_t)n * s.C_out + (size_t)g * s.Kg + (size_t)nt * Kt) * HW + f;
+            float* yk = y + ((size_t)n * s.C_out + (size_t)g * s.Kg + (size_t)nt * Kt) * OHW + fo;
             for (int k0 = 0; k0 < Kt; k0 += 8) {
                 float d0[8], d1[8], d2[8];
                 tmem_ld8(t0 + (uint32_t)k0, d0);
@@ -311,7 +320,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                         if (lane == 31) xchg[buf][wq][0][k0 + i] = d0[i];
                         if (lane == 0) xchg[buf][wq][1][k0 + i] = d2[i];
                     }
-                    if (valid) yk[(size_t)(k0 + i) * HW] = v;
+                    if (valid) yk[(size_t)(k0 + i) * OHW] = v;
                 }
             }
             tc_fence_before();
@@ -323,9 +332,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg_bar[buf]));
                 if (!mbar_wait(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
                 if (valid && lane == 0 && wq > 0 && use_left)
-                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * HW] += xchg[buf][wq - 1][0][k];
+                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * OHW] += xchg[buf][wq - 1][0][k];
                 if (valid && lane == 31 && wq < 3 && use_right)
-                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * HW] += xchg[buf][wq + 1][1][k];
+                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * OHW] += xchg[buf][wq + 1][1][k];
             }
         }
     }
@@ -393,7 +402,7 @@ EncodeTiledFn get_encode_fn() {
 }  // namespace
 
 bool igemm_supported(const Shape& s) {
-    if (!(s.KH == 3 && s.KW == 3 && s.stride == 1 && s.pad == 1 && s.dilation == 1)) return false;
+    if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.pad == 1 && s.dilation == 1)) return false;
     if (s.Cg % 8 != 0 || s.Kg % 8 != 0) return false;
     if (s.W % 4 != 0 || s.W > 128) return false;
     if ((long long)s.H * s.W < 32) return false;
@@ -412,8 +421,13 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
     c.Np = (3 * kt + 15) & ~15;
     const int HW = s.H * s.W;
     c.seg_mode = (32 % s.W == 0) && (HW % 32 == 0);
+    c.seg_fstep = 32;
     if (c.seg_mode) {
         c.SPI = HW / 32;
+        if (s.stride == 2 && s.W == 32) {   // a segment is one row: visit the even rows only
+            c.seg_fstep = 64;
+            c.SPI = (s.H + 1) / 2;
+        }
         c.R = 0;
         c.RB = 0;
         c.MT = (int)(((long long)s.N * c.SPI + 3) / 4);

@@ -62,6 +62,8 @@ ODD_SHAPES = [
     (1, 6, 15, 15, 6, 3, 3, 1, 2, 2, 2), (2, 32, 16, 16, 32, 3, 3, 1, 1, 1, 2), (1, 48, 20, 24, 96, 3, 3, 1, 1, 1, 3),
     (2, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1), (1, 32, 7, 7, 32, 3, 3, 1, 1, 1, 1), (1, 24, 56, 56, 24, 3, 3, 2, 1, 1, 24),
     (5, 3, 37, 41, 3, 3, 3, 1, 1, 1, 3), (1, 4, 64, 130, 4, 3, 3, 1, 1, 1, 4), (2, 16, 33, 35, 16, 3, 3, 2, 1, 1, 4),
+    (2, 16, 33, 36, 24, 3, 3, 2, 1, 1, 2), (1, 32, 31, 32, 32, 3, 3, 2, 1, 1, 1), (3, 8, 16, 16, 16, 3, 3, 2, 1, 1, 1),
+    (1, 64, 9, 64, 64, 3, 3, 2, 1, 1, 4), (2, 96, 10, 8, 96, 3, 3, 1, 1, 1, 1), (1, 128, 6, 128, 128, 3, 3, 1, 1, 1, 2),
     (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
 ]
 
