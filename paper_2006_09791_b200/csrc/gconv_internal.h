@@ -81,13 +81,18 @@ cudaError_t tiled_forward(const Shape& s, const float* x, const void* packed, fl
 
 // IGEMM_TF32: tile geometry of the tcgen05 implicit-GEMM kernel.
 struct IgemmCfg {
+    int merge, groups, Cg, Kg;   // adjacent groups presented as one (block-diagonal filters); sizes after merging
     int CK, chunks;          // channels per pipeline stage, stages per vertical tap
+    int nr, nseg, wseg;      // vertical taps served by one stage (1 or 3), segments per stage, segments per image row
+    int b_res;               // weights of a (group, filter tile) stay resident in shared memory
+    uint32_t bres_stride;    // bytes between the two resident weight buffers
     int Kt, NT, Np;          // filters per tile, filter tiles per group, MMA N (3*Kt padded to 16)
     int seg_mode;            // 1: a tile is any four 32-pixel segments (W divides 32); 0: a tile is R whole rows
     int SPI, R, RB, MT;      // segments per image; rows per tile, row blocks per image; pixel tiles in total
     int seg_fstep;           // flat-pixel step between consecutive segments of an image
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int num_tiles, stages, grid;
+    FastDiv div_mt, div_spi, div_w;   // tile -> (group/filter tile, pixel tile); pixel tile -> (image, segment or row block); pixel -> (row, column)
     uint32_t stage_bytes;
     size_t smem_bytes;
 };

@@ -27,7 +27,7 @@
 // (group, filter tile, pixel tile), one CTA per SM walks it.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + single-thread MMA issuer,
-// warps 2..5 = epilogue (TMEM lane quarter = warp_id % 4).  Every mbarrier wait is bounded: when a
+// warps 2..9 = epilogue (TMEM lane quarter = warp_id % 4, two warps per quarter split the filters).  Every mbarrier wait is bounded: when a
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
 // copies are waited for (bounded), TMEM is freed and the kernel returns.
 #include <cuda.h>
@@ -38,7 +38,8 @@ namespace gconv {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each takes half of the filters
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;          // TMEM column offset between the two accumulator buffers
 constexpr uint32_t kSpinLimit = 1u << 20;
@@ -49,6 +50,8 @@ struct __align__(8) SharedCtl {
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
     unsigned long long xchg_bar[2];
+    unsigned long long b_full[2];   // resident weights of a (group, filter tile) have landed
+    unsigned long long b_free[2];   // every MMA that read that weight buffer has completed
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -87,6 +90,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     record_status(status, GCONV_ERR_TIMEOUT, where);
     return false;
+}
+
+// The same wait for a converged warp: every lane gets the same answer, so the warp never splits
+// around the warp-level primitives that follow.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, Status* status,
+                                               int where) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, where) ? 1 : 0) != 0;
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
@@ -161,8 +171,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl.tmem_full[i]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[i]), 4);
-            mbar_init(smem_u32(&ctl.xchg_bar[i]), 4);
+            mbar_init(smem_u32(&ctl.tmem_empty[i]), kEpiWarps);
+            mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
+            mbar_init(smem_u32(&ctl.b_full[i]), 1);
+            mbar_init(smem_u32(&ctl.b_free[i]), 1);
         }
         ctl.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -178,61 +190,91 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
 
-    const int kstages = 3 * c.chunks;                 // pipeline stages per tile: (r, channel chunk)
-    const uint32_t a_bytes = 4u * (uint32_t)c.CK * 128u;
-    const uint32_t b_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;
+    // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
+    // segments of one vertical tap (nr = 1, stages run chunk-major, tap-minor), or the tile plus its
+    // row halo (nr = 3: the three taps are views of the same stage, shifted by whole segments).
+    const int kstages = (3 / c.nr) * c.chunks;
+    const uint32_t seg_bytes = (uint32_t)c.CK * 128u;
+    const uint32_t a_bytes = (uint32_t)c.nseg * seg_bytes;
+    const uint32_t blk_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;   // weights of one (chunk, tap)
+    const uint32_t b_tile_bytes = 3u * (uint32_t)c.chunks * blk_bytes;   // weights of one (group, filter tile)
+    const uint32_t bres_base = smem_base;                                // two resident weight buffers (if b_res)
+    const uint32_t stage_base = smem_base + (c.b_res ? 2u * c.bres_stride : 0u);
     const int HW = s.H * s.W;
     const size_t OHW = (size_t)s.H_out * s.W_out;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
-                const int mt = tile % c.MT;
-                const int rest = tile / c.MT;
-                const int nt = rest % c.NT;
-                const int g = rest / c.NT;
-                int seg_n[4], seg_f[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (c.seg_mode) {
-                        const int sg = mt * 4 + j;
-                        int n = sg / c.SPI;
-                        seg_f[j] = (sg - n * c.SPI) * c.seg_fstep;
-                        seg_n[j] = n < s.N ? n : s.N;   // past the last image: fully out of bounds, zero fill
-                    } else {
-                        const int n = mt / c.RB;
-                        seg_n[j] = n;
-                        seg_f[j] = (mt - n * c.RB) * c.R * s.W + 32 * j;
-                    }
-                }
-                const uint8_t* wtile = wblocks + (size_t)(g * c.NT + nt) * (size_t)kstages * b_bytes;
-                for (int ks = 0; ks < kstages; ++ks, ++it) {
-                    const int stage = it % c.stages;
-                    const uint32_t ph = (it / c.stages) & 1;
-                    if (!mbar_wait(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
-                    const int r = ks / c.chunks;
-                    const int ch = ks - r * c.chunks;
-                    const uint32_t full = smem_u32(&ctl.full[stage]);
-                    const uint32_t a_dst = smem_base + (uint32_t)stage * c.stage_bytes;
-                    mbar_arrive_expect_tx(full, a_bytes + b_bytes);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        tma_load_3d(a_dst + (uint32_t)j * (uint32_t)c.CK * 128u, &xmap, seg_f[j] + (r - 1) * s.W,
-                                    g * s.Cg + ch * c.CK, seg_n[j], full);
-                    bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * b_bytes, b_bytes, full);
-                }
+        // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
+        uint32_t it = 0, switches = 0;
+        int cur_gn = -1;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
+            uint32_t gn, mt;
+            c.div_mt.divmod((uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
+            const int g = (int)gn / c.NT;
+            const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
+            if (c.b_res && (int)gn != cur_gn) {
+                const uint32_t bb = switches & 1, use = switches >> 1;
+                if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
+                const uint32_t bar = smem_u32(&ctl.b_full[bb]);
+                if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
+                __syncwarp();
+                for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                    bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
+                cur_gn = (int)gn;
+                ++switches;
             }
-            if (!ok) {
-                // drain: wait (bounded) for the copies of every stage that may still be in flight
-                for (int i = 0; i < c.stages && i < (int)it; ++i) {
-                    const uint32_t j = it - 1 - i;
-                    const uint32_t bar = smem_u32(&ctl.full[j % c.stages]);
-                    for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
-                        if (mbar_try_wait(bar, (j / c.stages) & 1)) break;
+            // this lane's segment: image index and first flat pixel (tap r adds (r-1)*W)
+            int my_n, my_f;
+            if (c.nr == 3) {                               // tile plus halo: contiguous segments of one image
+                uint32_t n, i;
+                if (c.seg_mode) c.div_spi.divmod(mt * 4u, n, i); else c.div_spi.divmod(mt, n, i);
+                my_n = (int)n;
+                my_f = (c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W) + (lane - c.wseg) * 32;
+            } else if (c.seg_mode) {
+                uint32_t n, i;
+                c.div_spi.divmod(mt * 4u + (uint32_t)(lane & 3), n, i);
+                my_n = (int)n < s.N ? (int)n : s.N;        // past the last image: fully out of bounds, zero fill
+                my_f = (int)i * c.seg_fstep;
+            } else {
+                uint32_t n, i;
+                c.div_spi.divmod(mt, n, i);
+                my_n = (int)n;
+                my_f = (int)i * c.R * s.W + 32 * (lane & 3);
+            }
+            const bool issuer = lane < c.nseg;
+            for (int ks = 0; ks < kstages; ++ks, ++it) {
+                const int stage = it % c.stages;
+                const uint32_t ph = (it / c.stages) & 1;
+                if (!mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                const uint32_t full = smem_u32(&ctl.full[stage]);
+                const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
+                const int ch = c.nr == 3 ? ks : ks / 3;
+                const int r = c.nr == 3 ? 1 : ks - ch * 3;
+                const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(full, a_bytes + nb);
+                    if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
                 }
+                __syncwarp();
+                if (issuer)
+                    tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, g * c.Cg + ch * c.CK, my_n, full);
+            }
+        }
+        if (!ok && lane == 0) {
+            // drain: wait (bounded) for the copies of every stage that may still be in flight
+            for (int i = 0; i < c.stages && i < (int)it; ++i) {
+                const uint32_t j = it - 1 - i;
+                const uint32_t bar = smem_u32(&ctl.full[j % c.stages]);
+                for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
+                    if (mbar_try_wait(bar, (j / c.stages) & 1)) break;
+            }
+            for (uint32_t i = 0; i < 2 && i < switches; ++i) {
+                const uint32_t j = switches - 1 - i;
+                const uint32_t bar = smem_u32(&ctl.b_full[j & 1]);
+                for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
+                    if (mbar_try_wait(bar, (j >> 1) & 1)) break;
             }
         }
     } else if (warp == 1) {
@@ -240,26 +282,53 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((uint32_t)(c.Np >> 3) << 17) |
                                    ((128u >> 4) << 24);
-            const uint32_t a_lbo = (uint32_t)c.CK * 128u;          // next 32-pixel block
             const uint32_t b_lbo = (uint32_t)(c.Np >> 3) * 128u;   // next 4-channel core matrix along K
             const uint32_t b_kstep = 2u * b_lbo;                   // 8 channels
-            uint32_t it = 0, tcount = 0;
+            // descriptors differ only in the start-address field of the low word
+            const uint64_t a_hi = make_desc(0, seg_bytes, 512u, 1u);
+            const uint64_t b_hi = make_desc(0, b_lbo, 128u, 0u);
+            const int k8n = c.CK / 8;
+            uint32_t it = 0, tcount = 0, switches = 0;
+            int cur_gn = -1;
+            uint32_t bres_addr = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x, ++tcount) {
+                uint32_t gn, mt;
+                c.div_mt.divmod((uint32_t)tile, gn, mt);
+                if (c.b_res && (int)gn != cur_gn) {
+                    // the previous weight buffer is free once every MMA issued so far has completed
+                    if (switches > 0) umma_commit(smem_u32(&ctl.b_free[(switches - 1) & 1]));
+                    const uint32_t bb = switches & 1, use = switches >> 1;
+                    if (!mbar_wait(smem_u32(&ctl.b_full[bb]), use & 1, abort_flag, status, 700 + bb)) break;
+                    bres_addr = bres_base + bb * c.bres_stride;
+                    cur_gn = (int)gn;
+                    ++switches;
+                }
                 const uint32_t buf = tcount & 1;
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag, status, 200 + buf)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                uint32_t acc = 0;
                 for (int ks = 0; ks < kstages; ++ks, ++it) {
                     const int stage = it % c.stages;
                     if (!mbar_wait(smem_u32(&ctl.full[stage]), (it / c.stages) & 1, abort_flag, status, 300 + stage)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + (uint32_t)stage * c.stage_bytes;
-                    const uint32_t b_addr = a_addr + a_bytes;
-                    for (int k8 = 0; k8 < c.CK / 8; ++k8) {
-                        const uint64_t adesc = make_desc(a_addr + (uint32_t)k8 * 1024u, a_lbo, 512u, 1u);
-                        const uint64_t bdesc = make_desc(b_addr + (uint32_t)k8 * b_kstep, b_lbo, 128u, 0u);
-                        umma_tf32(d_tmem, adesc, bdesc, idesc, (ks | k8) != 0 ? 1u : 0u);
+                    const uint32_t a_addr = stage_base + (uint32_t)stage * c.stage_bytes;
+                    for (int rr = 0; rr < c.nr; ++rr) {
+                        // tap r: with a halo stage it is the view that starts r rows (wseg segments per row) in
+                        const uint32_t a_view = a_addr + (c.nr == 3 ? (uint32_t)(rr * c.wseg) * seg_bytes : 0u);
+                        const uint32_t blk = c.nr == 3 ? (uint32_t)(ks * 3 + rr) : (uint32_t)ks;   // (chunk, tap) block
+                        const uint32_t b_addr = c.b_res ? bres_addr + blk * blk_bytes
+                                                        : a_addr + a_bytes + (c.nr == 3 ? (uint32_t)rr * blk_bytes : 0u);
+                        uint64_t adesc = a_hi | (uint64_t)((a_view >> 4) & 0x3FFFu);
+                        uint64_t bdesc = b_hi | (uint64_t)((b_addr >> 4) & 0x3FFFu);
+#pragma unroll 4
+                        for (int k8 = 0; k8 < k8n; ++k8) {
+                            umma_tf32(d_tmem, adesc, bdesc, idesc, acc);
+                            acc = 1;
+                            adesc += 1024u >> 4;
+                            bdesc += b_kstep >> 4;
+                        }
                     }
                     umma_commit(smem_u32(&ctl.empty[stage]));
                 }
@@ -269,72 +338,79 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int wq = warp & 3;                       // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;              // which half of the tile's filters this warp stores
         const int l = wq * 32 + lane;                  // pixel lane inside the tile
         const int Kt = c.Kt;
+        const int kh = (Kt / 2 + 7) & ~7;              // filters of the first half (multiple of 8)
+        const int kbeg = half == 0 ? 0 : kh;
+        const int kend = half == 0 ? kh : Kt;
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < c.num_tiles; tile += gridDim.x, ++tcount) {
-            const int mt = tile % c.MT;
-            const int rest = tile / c.MT;
-            const int nt = rest % c.NT;
-            const int g = rest / c.NT;
-            int n, f;
+            uint32_t gn, mt;
+            c.div_mt.divmod((uint32_t)tile, gn, mt);
+            uint32_t n, i;
+            int f;
             bool valid;
             if (c.seg_mode) {
-                const int sg = mt * 4 + wq;
-                n = sg / c.SPI;
-                f = (sg - n * c.SPI) * c.seg_fstep + lane;
-                valid = n < s.N;
+                c.div_spi.divmod(mt * 4u + (uint32_t)wq, n, i);
+                f = (int)i * c.seg_fstep + lane;
+                valid = (int)n < s.N;
             } else {
-                n = mt / c.RB;
-                f = (mt - n * c.RB) * c.R * s.W + l;
+                c.div_spi.divmod(mt, n, i);
+                f = (int)i * c.R * s.W + l;
                 valid = (l < c.R * s.W) && (f < HW);
             }
-            const int prow = f / s.W;
-            const int q = f - prow * s.W;
+            uint32_t prow, q;
+            c.div_w.divmod((uint32_t)f, prow, q);
             const bool use_left = q > 0;
-            const bool use_right = q < s.W - 1;
+            const bool use_right = (int)q < s.W - 1;
             int fo = f;                                  // position in the output plane
             if (s.stride == 2) {                         // stride 2 keeps the even rows and columns of the stride-1 result
                 valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
-                fo = (prow >> 1) * s.W_out + (q >> 1);
+                fo = (int)(prow >> 1) * s.W_out + (int)(q >> 1);
             }
+            const bool add_up = use_left && lane > 0;
+            const bool add_dn = use_right && lane < 31;
             const uint32_t buf = tcount & 1;
-            if (!mbar_wait(smem_u32(&ctl.tmem_full[buf]), (tcount >> 1) & 1, abort_flag, status, 400 + buf)) break;
+            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), (tcount >> 1) & 1, abort_flag, status, 400 + buf)) break;
             tc_fence_after();
             const uint32_t t0 = tmem_base + buf * kAccStride + ((uint32_t)(wq * 32) << 16);
-            float* yk = y + ((size_t)n * s.C_out + (size_t)g * s.Kg + (size_t)nt * Kt) * OHW + fo;
-            for (int k0 = 0; k0 < Kt; k0 += 8) {
+            // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
+            float* yk0 = y + ((size_t)n * s.C_out + (size_t)gn * Kt) * OHW + fo;
+            float* yk = yk0 + (size_t)kbeg * OHW;
+            for (int k0 = kbeg; k0 < kend; k0 += 8) {
                 float d0[8], d1[8], d2[8];
                 tmem_ld8(t0 + (uint32_t)k0, d0);
                 tmem_ld8(t0 + (uint32_t)(Kt + k0), d1);
                 tmem_ld8(t0 + (uint32_t)(2 * Kt + k0), d2);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float up = __shfl_up_sync(0xffffffffu, d0[i], 1);
-                    const float dn = __shfl_down_sync(0xffffffffu, d2[i], 1);
-                    float v = d1[i];
-                    if (use_left && lane > 0) v += up;
-                    if (use_right && lane < 31) v += dn;
+                for (int j = 0; j < 8; ++j) {
+                    const float up = __shfl_up_sync(0xffffffffu, d0[j], 1);
+                    const float dn = __shfl_down_sync(0xffffffffu, d2[j], 1);
+                    float v = d1[j];
+                    if (add_up) v += up;
+                    if (add_dn) v += dn;
                     if (c.need_xchg) {
-                        if (lane == 31) xchg[buf][wq][0][k0 + i] = d0[i];
-                        if (lane == 0) xchg[buf][wq][1][k0 + i] = d2[i];
+                        if (lane == 31) xchg[buf][wq][0][k0 + j] = d0[j];
+                        if (lane == 0) xchg[buf][wq][1][k0 + j] = d2[j];
                     }
-                    if (valid) yk[(size_t)(k0 + i) * OHW] = v;
+                    if (valid) *yk = v;
+                    yk += OHW;
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
             if (c.need_xchg) {
-                // rows that straddle a warp boundary: add the neighbour warp's edge lane once all four
+                // rows that straddle a warp boundary: add the neighbour warp's edge lane once all
                 // epilogue warps have published theirs (bounded mbarrier wait, never a named barrier)
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg_bar[buf]));
-                if (!mbar_wait(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
+                if (!mbar_wait_warp(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
                 if (valid && lane == 0 && wq > 0 && use_left)
-                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * OHW] += xchg[buf][wq - 1][0][k];
+                    for (int k = kbeg; k < kend; ++k) yk0[(size_t)k * OHW] += xchg[buf][wq - 1][0][k];
                 if (valid && lane == 31 && wq < 3 && use_right)
-                    for (int k = 0; k < Kt; ++k) yk[(size_t)k * OHW] += xchg[buf][wq + 1][1][k];
+                    for (int k = kbeg; k < kend; ++k) yk0[(size_t)k * OHW] += xchg[buf][wq + 1][1][k];
             }
         }
     }
@@ -347,12 +423,14 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
     }
 }
 
-// Weight pre-pack for this variant.  Output block (g, nt, r, chunk) is the shared-memory image of
-// the K-major, unswizzled B operand of one pipeline stage: [k8][k2][n/8][n%8][4 channels], where
-// column n = s*Kt + k holds filter nt*Kt + k at horizontal tap s (columns >= 3*Kt are zero) and
-// values are rounded to TF32 (round to nearest, ties away from zero).
+// Weight pre-pack for this variant.  Output block (group, filter tile, chunk, r) is the shared-memory
+// image of the K-major, unswizzled B operand of one (channel chunk, vertical tap):
+// [k8][k2][n/8][n%8][4 channels], where column n = s*Kt + k holds filter k of the tile at horizontal
+// tap s (columns >= 3*Kt are zero) and values are rounded to TF32 (round to nearest, ties away).
+// When `merge` > 1 that many adjacent groups are presented to the kernel as one group with a
+// block-diagonal filter bank: entries that would mix channels of different groups are zero.
 __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__ w, uint32_t* __restrict__ packed, uint32_t tag) {
-    const size_t total = (size_t)s.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         packed[0] = tag;
@@ -366,18 +444,22 @@ __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__
         const int nb = (int)(t % (c.Np / 8)); t /= (c.Np / 8);
         const int k2 = (int)(t % 2); t /= 2;
         const int k8 = (int)(t % (c.CK / 8)); t /= (c.CK / 8);
-        const int ch = (int)(t % c.chunks); t /= c.chunks;
         const int r = (int)(t % 3); t /= 3;
+        const int ch = (int)(t % c.chunks); t /= c.chunks;
         const int nt = (int)(t % c.NT);
-        const int g = (int)(t / c.NT);
+        const int g = (int)(t / c.NT);             // merged group
         const int ncol = nb * 8 + n8;
-        const int cc = ch * c.CK + k8 * 8 + k2 * 4 + e;
+        const int ce = ch * c.CK + k8 * 8 + k2 * 4 + e;   // channel within the merged group
         uint32_t bits = 0;
         if (ncol < 3 * c.Kt) {
             const int ss = ncol / c.Kt;
-            const int k = ncol - ss * c.Kt;
-            const float v = w[(((size_t)(g * s.Kg + nt * c.Kt + k)) * s.Cg + cc) * 9 + r * 3 + ss];
-            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(bits) : "f"(v));
+            const int ke = nt * c.Kt + (ncol - ss * c.Kt);  // filter within the merged group
+            const int gi = ke / s.Kg;                        // which original group of the merge
+            if (ce / s.Cg == gi) {
+                const int ko = (g * c.merge + gi) * s.Kg + (ke - gi * s.Kg);
+                const float v = w[(((size_t)ko) * s.Cg + (ce - gi * s.Cg)) * 9 + r * 3 + ss];
+                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(bits) : "f"(v));
+            }
         }
         dst[i] = bits;
     }
@@ -401,9 +483,16 @@ EncodeTiledFn get_encode_fn() {
 
 }  // namespace
 
+static int igemm_merge(const Shape& s) {
+    int m = 1;
+    while (m * 2 <= s.groups && s.groups % (m * 2) == 0 && s.Cg * m * 2 <= 32 && s.Kg * m * 2 <= 64) m *= 2;
+    return m;
+}
+
 bool igemm_supported(const Shape& s) {
     if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.pad == 1 && s.dilation == 1)) return false;
-    if (s.Cg % 8 != 0 || s.Kg % 8 != 0) return false;
+    const int m = igemm_merge(s);
+    if ((s.Cg * m) % 8 != 0 || (s.Kg * m) % 8 != 0) return false;
     if (s.W % 4 != 0 || s.W > 128) return false;
     if ((long long)s.H * s.W < 32) return false;
     if (s.C_in > 65535 * 8) return false;
@@ -412,12 +501,16 @@ bool igemm_supported(const Shape& s) {
 
 IgemmCfg igemm_config(const Shape& s, int sm_count) {
     IgemmCfg c;
-    c.CK = (s.Cg % 32 == 0) ? 32 : (s.Cg % 16 == 0 ? 16 : 8);
-    c.chunks = s.Cg / c.CK;
-    int kt = s.Kg <= 64 ? s.Kg : 64;
-    while (s.Kg % kt != 0 || kt % 8 != 0) kt -= 8;   // largest multiple of 8 dividing Kg, at most 64
+    c.merge = igemm_merge(s);
+    c.groups = s.groups / c.merge;
+    c.Cg = s.Cg * c.merge;
+    c.Kg = s.Kg * c.merge;
+    c.CK = (c.Cg % 32 == 0) ? 32 : (c.Cg % 16 == 0 ? 16 : 8);
+    c.chunks = c.Cg / c.CK;
+    int kt = c.Kg <= 64 ? c.Kg : 64;
+    while (c.Kg % kt != 0 || kt % 8 != 0) kt -= 8;   // largest multiple of 8 dividing Kg, at most 64
     c.Kt = kt;
-    c.NT = s.Kg / kt;
+    c.NT = c.Kg / kt;
     c.Np = (3 * kt + 15) & ~15;
     const int HW = s.H * s.W;
     c.seg_mode = (32 % s.W == 0) && (HW % 32 == 0);
@@ -439,26 +532,44 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
         c.MT = s.N * c.RB;
         c.need_xchg = 1;
     }
-    c.num_tiles = s.groups * c.NT * c.MT;
-    const uint32_t a_bytes = 4u * c.CK * 128u, b_bytes = (uint32_t)c.Np * c.CK * 4u;
-    c.stage_bytes = (a_bytes + b_bytes + 1023u) & ~1023u;
-    int st = (int)((160u * 1024u) / c.stage_bytes);
+    // Row halo: when a row is a whole number of 32-pixel segments the three vertical taps are views of
+    // one staged block (tile + one row above and below), so the input crosses L2 -> shared memory once.
+    c.nr = 1;
+    c.nseg = 4;
+    c.wseg = 0;
+    if (s.stride == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
+        c.nr = 3;
+        c.wseg = s.W / 32;
+        c.nseg = 4 + 2 * c.wseg;
+    }
+    c.num_tiles = c.groups * c.NT * c.MT;
+    c.div_mt = make_fastdiv((uint32_t)c.MT);
+    c.div_spi = make_fastdiv((uint32_t)(c.seg_mode ? c.SPI : c.RB));
+    c.div_w = make_fastdiv((uint32_t)s.W);
+    const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
+    const uint32_t b_tile = 3u * c.chunks * blk;
+    c.b_res = b_tile <= 40u * 1024u ? 1 : 0;          // keep a (group, filter tile)'s weights resident, double buffered
+    c.bres_stride = (b_tile + 1023u) & ~1023u;
+    const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
+    c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
+    const uint32_t budget = 196u * 1024u - (c.b_res ? 2u * c.bres_stride : 0u);
+    int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
     if (st < 2) st = 2;
     c.stages = st;
-    c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024;
+    c.smem_bytes = (size_t)c.stages * c.stage_bytes + (c.b_res ? 2u * c.bres_stride : 0u) + 1024;
     c.grid = c.num_tiles < sm_count ? c.num_tiles : sm_count;
     return c;
 }
 
 size_t igemm_packed_bytes(const Shape& s) {
     const IgemmCfg c = igemm_config(s, 148);
-    return kHeaderBytes + sizeof(float) * (size_t)s.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    return kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
 }
 
 cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_t st) {
     const IgemmCfg c = igemm_config(s, 148);
-    const size_t total = (size_t)s.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
     int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
     igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
     return cudaGetLastError();
@@ -483,7 +594,7 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(igemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(igemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
