@@ -92,6 +92,7 @@ struct IgemmCfg {
     int seg_fstep;           // flat-pixel step between consecutive segments of an image
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int num_tiles, stages, grid;
+    FastDiv div_nt;                   // (group, filter tile) index -> group
     FastDiv div_mt, div_spi, div_w;   // tile -> (group/filter tile, pixel tile); pixel tile -> (image, segment or row block); pixel -> (row, column)
     uint32_t stage_bytes;
     size_t smem_bytes;

@@ -207,12 +207,17 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
         // ---------------------------------------------------------------- TMA producer
         // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
         uint32_t it = 0, switches = 0;
+        int stage = 0;
+        uint32_t ph = 0;                                   // phase parity of the current pass over the stage ring
         int cur_gn = -1;
         bool ok = true;
+        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
         for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
             uint32_t gn, mt;
             c.div_mt.divmod((uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
-            const int g = (int)gn / c.NT;
+            uint32_t gq, ntq;
+            c.div_nt.divmod(gn, gq, ntq);
+            const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
             if (c.b_res && (int)gn != cur_gn) {
                 const uint32_t bb = switches & 1, use = switches >> 1;
@@ -244,14 +249,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 my_f = (int)i * c.R * s.W + 32 * (lane & 3);
             }
             const bool issuer = lane < c.nseg;
+            int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
-                const int stage = it % c.stages;
-                const uint32_t ph = (it / c.stages) & 1;
                 if (!mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
-                const int ch = c.nr == 3 ? ks : ks / 3;
-                const int r = c.nr == 3 ? 1 : ks - ch * 3;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
                 if (lane == 0) {
                     mbar_arrive_expect_tx(full, a_bytes + nb);
@@ -260,6 +262,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 __syncwarp();
                 if (issuer)
                     tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, g * c.Cg + ch * c.CK, my_n, full);
+                if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
+                if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
         }
         if (!ok && lane == 0) {
@@ -288,7 +292,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             const uint64_t a_hi = make_desc(0, seg_bytes, 512u, 1u);
             const uint64_t b_hi = make_desc(0, b_lbo, 128u, 0u);
             const int k8n = c.CK / 8;
-            uint32_t it = 0, tcount = 0, switches = 0;
+            uint32_t tcount = 0, switches = 0;
+            int stage = 0;
+            uint32_t ph = 0;
             int cur_gn = -1;
             uint32_t bres_addr = 0;
             bool ok = true;
@@ -309,9 +315,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * kAccStride;
                 uint32_t acc = 0;
-                for (int ks = 0; ks < kstages; ++ks, ++it) {
-                    const int stage = it % c.stages;
-                    if (!mbar_wait(smem_u32(&ctl.full[stage]), (it / c.stages) & 1, abort_flag, status, 300 + stage)) { ok = false; break; }
+                for (int ks = 0; ks < kstages; ++ks) {
+                    if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 300 + stage)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = stage_base + (uint32_t)stage * c.stage_bytes;
                     for (int rr = 0; rr < c.nr; ++rr) {
@@ -331,6 +336,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                         }
                     }
                     umma_commit(smem_u32(&ctl.empty[stage]));
+                    if (++stage == c.stages) { stage = 0; ph ^= 1; }
                 }
                 if (ok) umma_commit(smem_u32(&ctl.tmem_full[buf]));
             }
@@ -376,8 +382,28 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             tc_fence_after();
             const uint32_t t0 = tmem_base + buf * kAccStride + ((uint32_t)(wq * 32) << 16);
             // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
-            float* yk0 = y + ((size_t)n * s.C_out + (size_t)gn * Kt) * OHW + fo;
-            float* yk = yk0 + (size_t)kbeg * OHW;
+            float* yk = y + ((size_t)n * s.C_out + (size_t)gn * Kt + (size_t)kbeg) * OHW + fo;
+            if (c.need_xchg) {
+                // Rows may straddle a warp boundary: publish this warp's edge lanes (lane 31's left-tap
+                // and lane 0's right-tap accumulators) so the neighbouring quarter can add them, then wait
+                // (bounded mbarrier wait, never a named barrier) until all epilogue warps have published.
+                for (int k0 = kbeg; k0 < kend; k0 += 8) {
+                    float d0[8], d2[8];
+                    tmem_ld8(t0 + (uint32_t)k0, d0);
+                    tmem_ld8(t0 + (uint32_t)(2 * Kt + k0), d2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (lane == 31) xchg[buf][wq][0][k0 + j] = d0[j];
+                        if (lane == 0) xchg[buf][wq][1][k0 + j] = d2[j];
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg_bar[buf]));
+                if (!mbar_wait_warp(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
+            }
+            const bool edge_up = c.need_xchg && lane == 0 && wq > 0 && use_left;     // left neighbour is in the previous quarter
+            const bool edge_dn = c.need_xchg && lane == 31 && wq < 3 && use_right;   // right neighbour is in the next quarter
             for (int k0 = kbeg; k0 < kend; k0 += 8) {
                 float d0[8], d1[8], d2[8];
                 tmem_ld8(t0 + (uint32_t)k0, d0);
@@ -391,10 +417,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                     float v = d1[j];
                     if (add_up) v += up;
                     if (add_dn) v += dn;
-                    if (c.need_xchg) {
-                        if (lane == 31) xchg[buf][wq][0][k0 + j] = d0[j];
-                        if (lane == 0) xchg[buf][wq][1][k0 + j] = d2[j];
-                    }
+                    if (edge_up) v += xchg[buf][wq - 1][0][k0 + j];
+                    if (edge_dn) v += xchg[buf][wq + 1][1][k0 + j];
                     if (valid) *yk = v;
                     yk += OHW;
                 }
@@ -402,16 +426,6 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
-            if (c.need_xchg) {
-                // rows that straddle a warp boundary: add the neighbour warp's edge lane once all
-                // epilogue warps have published theirs (bounded mbarrier wait, never a named barrier)
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg_bar[buf]));
-                if (!mbar_wait_warp(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
-                if (valid && lane == 0 && wq > 0 && use_left)
-                    for (int k = kbeg; k < kend; ++k) yk0[(size_t)k * OHW] += xchg[buf][wq - 1][0][k];
-                if (valid && lane == 31 && wq < 3 && use_right)
-                    for (int k = kbeg; k < kend; ++k) yk0[(size_t)k * OHW] += xchg[buf][wq + 1][1][k];
-            }
         }
     }
 
@@ -546,6 +560,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
     c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)(c.seg_mode ? c.SPI : c.RB));
     c.div_w = make_fastdiv((uint32_t)s.W);
+    c.div_nt = make_fastdiv((uint32_t)c.NT);
     const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
     const uint32_t b_tile = 3u * c.chunks * blk;
     c.b_res = b_tile <= 40u * 1024u ? 1 : 0;          // keep a (group, filter tile)'s weights resident, double buffered
