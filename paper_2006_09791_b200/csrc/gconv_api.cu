@@ -5,16 +5,6 @@
 
 using namespace gconv;
 
-struct gconv_desc {
-    Shape s;
-    int variant;         // resolved variant (never AUTO)
-    int forced;          // 1 if set by gconv_desc_set_variant
-    Status* status_dev;  // lazily allocated device status block
-    int device;          // device the status block lives on (-1 = none yet)
-    int sm_count;
-    int last_cuda_error;
-};
-
 namespace {
 
 bool variant_supported(const Shape& s, int v) {

@@ -7,14 +7,28 @@
 #include "../../include/gconv.h"
 
 namespace gconv {
-
-constexpr int kHeaderBytes = 64;  // packed-weight blob header; keeps the payload 16-byte aligned
-constexpr uint32_t kMagic = 0x47434e56u;  // "GCNV"
-
+struct Status;
 struct Shape {
     int N, C_in, H, W, C_out, KH, KW, stride, pad, dilation, groups;
     int Cg, Kg, H_out, W_out;
 };
+}  // namespace gconv
+
+// The descriptor behind gconv_desc_t.
+struct gconv_desc {
+    gconv::Shape s;
+    int variant;                 // resolved variant (never AUTO)
+    int forced;                  // 1 if set by gconv_desc_set_variant
+    gconv::Status* status_dev;   // lazily allocated device status block
+    int device;                  // device the status block lives on (-1 = none yet)
+    int sm_count;
+    int last_cuda_error;
+};
+
+namespace gconv {
+
+constexpr int kHeaderBytes = 64;  // packed-weight blob header; keeps the payload 16-byte aligned
+constexpr uint32_t kMagic = 0x47434e56u;  // "GCNV"
 
 // Device status block: word 0 = first error recorded by a kernel (0 = none), word 1 = detail.
 struct Status {
