@@ -47,7 +47,8 @@ enum gconv_status {
     GCONV_ERR_ALIGNMENT = 4,     /* a device pointer is not 16-byte aligned */
     GCONV_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed; see gconv_last_cuda_error */
     GCONV_ERR_PACK_MISMATCH = 6, /* device status: w_packed was packed for another shape or variant */
-    GCONV_ERR_TIMEOUT = 7        /* device status: a bounded wait inside a kernel ran out */
+    GCONV_ERR_TIMEOUT = 7,       /* device status: a bounded wait inside a kernel ran out */
+    GCONV_ERR_TOO_LARGE = 8      /* the layer does not fit the fixed scratch of gconv_forward_host_static */
 };
 
 /* Kernel variants.  The numeric tolerance of a result follows the variant that produced it:
@@ -135,6 +136,32 @@ int gconv_forward(gconv_desc_t desc, const float *x_nchw, const void *w_packed, 
  */
 int gconv_forward_host(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host,
                        float *x_stage, float *y_stage, void *stream);
+
+/*
+ * gconv_forward_host_static -- gconv_forward_host for callers that are not allowed to allocate
+ * device memory (no counterpart in the paper; it exists for deployment reasons only).  Think of a
+ * plugin living inside an application whose allocator owns the GPU, a service that fixes its memory
+ * at start-up, code running between stream-capture begin and end, or a loop that cannot take the
+ * device-wide synchronisation a cudaMalloc implies.  It calls no cudaMalloc/cudaFree and no
+ * allocating library routine: the status block and the staging room for x and y live in one
+ * static device array inside the library (16 MiB + 256 bytes, held by every GPU that loads the
+ * library until the process ends).
+ *   x_host    host, fp32 [N, C_in, H, W], read.
+ *   w_packed  device, from gconv_pack_weights on a descriptor of the same shape and variant.
+ *   y_host    host, fp32 [N, C_out, H_out, W_out], written.
+ * Limit: x and y, each rounded up to 256 bytes, must fit in 16 MiB together; larger layers return
+ * GCONV_ERR_TOO_LARGE and nothing is enqueued.
+ * The call enqueues clear-status, copy-in, the kernel of the descriptor's variant and copy-out on
+ * `stream`, then SYNCHRONISES the stream and returns GCONV_OK or the status the kernel recorded
+ * (GCONV_ERR_PACK_MISMATCH, GCONV_ERR_TIMEOUT); so when it returns, y_host is complete.
+ * The first call made with a given device current resolves the static array's device address for
+ * that device (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * All calls share the one array, which still holds the previous call's data: the status block is
+ * cleared and the staging regions are rewritten on every call, so results never depend on it, but
+ * calls that overlap on the GPU (two streams, two threads) race and must be serialised by the caller.
+ * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT (w_packed), GCONV_ERR_TOO_LARGE, GCONV_ERR_CUDA.
+ */
+int gconv_forward_host_static(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host, void *stream);
 
 /* Number of kernel launches one gconv_forward of this descriptor enqueues (for launch accounting). */
 int gconv_forward_launches(gconv_desc_t desc);

@@ -237,6 +237,7 @@ const char* gconv_status_string(int status) {
         case GCONV_ERR_CUDA: return "CUDA call failed";
         case GCONV_ERR_PACK_MISMATCH: return "packed weights do not match the descriptor";
         case GCONV_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+        case GCONV_ERR_TOO_LARGE: return "layer larger than the static scratch (x and y must fit in 16 MiB)";
         default: return "unknown status";
     }
 }

@@ -21,6 +21,7 @@ GCONV_ERR_ALIGNMENT = 4
 GCONV_ERR_CUDA = 5
 GCONV_ERR_PACK_MISMATCH = 6
 GCONV_ERR_TIMEOUT = 7
+GCONV_ERR_TOO_LARGE = 8
 
 GCONV_VARIANT_AUTO = 0
 GCONV_VARIANT_DIRECT_GENERIC = 1
@@ -44,6 +45,7 @@ _SIGNATURES = {
     "gconv_pack_weights": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "gconv_forward": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "gconv_forward_host": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "gconv_forward_host_static": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "gconv_forward_launches": (ctypes.c_int, [_vp]),
     "gconv_last_status": (ctypes.c_int, [_vp, _vp]),
     "gconv_last_cuda_error": (ctypes.c_int, [_vp]),
@@ -155,6 +157,13 @@ def gconv_forward(desc, x_nchw, w_packed, y_nchw, stream=None) -> None:
 def gconv_forward_host(desc, x_host, w_packed, y_host, x_stage, y_stage, stream=None) -> None:
     _check(load().gconv_forward_host(desc, _ptr(x_host), _ptr(w_packed), _ptr(y_host), _ptr(x_stage), _ptr(y_stage),
                                      _stream(stream)), "gconv_forward_host")
+
+
+def gconv_forward_host_static(desc, x_host, w_packed, y_host, stream=None) -> None:
+    """Host-buffer forward that allocates nothing (static device scratch, at most 16 MiB of x + y);
+    blocks until y_host is complete and raises on any status other than GCONV_OK."""
+    _check(load().gconv_forward_host_static(desc, _ptr(x_host), _ptr(w_packed), _ptr(y_host), _stream(stream)),
+           "gconv_forward_host_static")
 
 
 def gconv_forward_launches(desc) -> int:
