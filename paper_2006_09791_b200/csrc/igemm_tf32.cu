@@ -26,7 +26,7 @@
 // All groups and all images run in one persistent launch: the tile index enumerates
 // (group, filter tile, pixel tile), one CTA per SM walks it.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + single-thread MMA issuer,
+// Warp roles: warp 0 = TMA producer, warps 1 and 10 = single-thread MMA issuers for alternate tiles (warp 1 owns TMEM),
 // warps 2..9 = epilogue (TMEM lane quarter = warp_id % 4, two warps per quarter split the filters).  Every mbarrier wait is bounded: when a
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
 // copies are waited for (bounded), TMEM is freed and the kernel returns.
@@ -39,7 +39,8 @@ namespace gconv {
 namespace {
 
 constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each takes half of the filters
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the first is warp 1)
+constexpr int kThreads = 96 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;          // TMEM column offset between the two accumulator buffers
 constexpr uint32_t kSpinLimit = 1u << 20;
@@ -174,7 +175,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             mbar_init(smem_u32(&ctl.tmem_empty[i]), kEpiWarps);
             mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
             mbar_init(smem_u32(&ctl.b_full[i]), 1);
-            mbar_init(smem_u32(&ctl.b_free[i]), 1);
+            mbar_init(smem_u32(&ctl.b_free[i]), 2);
         }
         ctl.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -281,8 +282,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                     if (mbar_try_wait(bar, (j >> 1) & 1)) break;
             }
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
+    } else if (warp == 1 || warp == kMmaWarp2) {
+        // ---------------------------------------------------------------- MMA issuers
+        // Two warps issue alternate tiles (each owns one TMEM buffer), so the barrier waits and descriptor
+        // set-up of one tile hide behind the other warp's MMAs.  Both walk every tile to keep the stage ring
+        // and the weight-buffer switches in step.
+        const uint32_t mslot = warp == 1 ? 0u : 1u;
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((uint32_t)(c.Np >> 3) << 17) |
                                    ((128u >> 4) << 24);
@@ -301,14 +306,26 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x, ++tcount) {
                 uint32_t gn, mt;
                 c.div_mt.divmod((uint32_t)tile, gn, mt);
+                const bool mine = (tcount & 1) == mslot;
                 if (c.b_res && (int)gn != cur_gn) {
-                    // the previous weight buffer is free once every MMA issued so far has completed
+                    // the previous weight buffer is free once every MMA this warp issued so far has completed
+                    // (the barrier counts both issuing warps)
                     if (switches > 0) umma_commit(smem_u32(&ctl.b_free[(switches - 1) & 1]));
-                    const uint32_t bb = switches & 1, use = switches >> 1;
-                    if (!mbar_wait(smem_u32(&ctl.b_full[bb]), use & 1, abort_flag, status, 700 + bb)) break;
-                    bres_addr = bres_base + bb * c.bres_stride;
+                    // Both warps observe every fill of a weight buffer, in order, even when the tiles that
+                    // use it are the other warp's: a parity wait is only meaningful one phase at a time.
+                    if (!mbar_wait(smem_u32(&ctl.b_full[switches & 1]), (switches >> 1) & 1, abort_flag, status, 700)) break;
+                    bres_addr = bres_base + (switches & 1) * c.bres_stride;
                     cur_gn = (int)gn;
                     ++switches;
+                }
+                if (!mine) {
+                    // The other warp's tile: observe its stages' phases in order (no MMAs, no release) so that
+                    // this warp's own parity waits never alias a phase it has not seen.
+                    for (int ks = 0; ks < kstages && ok; ++ks) {
+                        if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 800 + stage)) ok = false;
+                        if (++stage == c.stages) { stage = 0; ph ^= 1; }
+                    }
+                    continue;
                 }
                 const uint32_t buf = tcount & 1;
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag, status, 200 + buf)) break;
