@@ -23,7 +23,7 @@ bool variant_supported(const Shape& s, int v) {
 // Variant selector.  Keyed on (Cg, Kg, H*W, N) like the tile-size choice the paper leaves to
 // autotuning (Section III-C); the thresholds come from measured timings of the forced variants.
 int select_variant(const Shape& s) {
-    if (igemm_supported(s) && s.Cg >= 8 && s.Kg >= 8) return GCONV_VARIANT_IGEMM_TF32;
+    if (igemm_supported(s) && s.Cg >= 2) return GCONV_VARIANT_IGEMM_TF32;
     if (tiled_supported(s)) return GCONV_VARIANT_DIRECT_TILED;
     return GCONV_VARIANT_DIRECT_GENERIC;
 }
