@@ -39,6 +39,9 @@ BATCH = 128
 CPU_SAMPLE_BATCH = 8      # batch of the reference arm's per-step sample
 CPU_LEG_BATCH = 32        # batch of the cpu_baseline leg of the GPU arm
 L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes one launch of the dominant kernel moves on average over the step, from the ncu capture summarised in
+# profiles/bench_wrn_stack_launch_list.md (reads only: ncu attributes the write-back of y to no kernel).
+NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.67e6}
 
 
 def load_peaks():
@@ -337,7 +340,7 @@ def run_ours(args):
 
     # ---- per-layer table (the metric proper) and roofline of the dominant kernel --------------------
     rows, extra = [], {}
-    if rank == 0:
+    if rank == 0 and not args.no_layers:
         seen = {}
         for g, L in plan:
             key = (L.name, g)
@@ -366,7 +369,10 @@ def run_ours(args):
             ach = dom["flops"] / (dom["ms"] * 1e-3) / 1e12
             roofline = {"bound": "tensor" if dom_v == gconv.GCONV_VARIANT_IGEMM_TF32 else "alu", "achieved": ach,
                         "peak": pipe_peak / 1e12, "unit": "TFLOP/s", "frac": ach / (pipe_peak / 1e12), "traffic": None}
+        roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(gconv.variant_name(dom_v))
         roofline.update({"kernel": gconv.variant_name(dom_v), "launches_per_step": dom["launches"],
+                         "algorithmic_bytes_per_launch": dom["bytes"] / dom["launches"],
+                         "avg_launch_us": 1e3 * dom["ms"] / dom["launches"],
                          "share_of_step": dom["ms"] / sum(a["ms"] for a in by_variant.values()),
                          "peak_source": peaks["source"]})
         extra["roofline"] = roofline
@@ -419,6 +425,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="also time the group-count sweep and ResNeXt-shaped layers")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-layers", action="store_true", help="skip the per-layer table (short runs under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
