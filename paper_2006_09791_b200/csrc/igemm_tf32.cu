@@ -18,7 +18,7 @@
 //   * B_r comes from the pre-packed weights (kernel-reshaping stage of Algorithm 1): already
 //     TF32-rounded and stored as the exact shared-memory image of a K-major core-matrix operand,
 //     so one bulk copy per pipeline stage stages it.
-//   * D lives in TMEM (3*Kt <= 192 fp32 columns, double buffered), the epilogue warps read it with
+//   * D lives in TMEM (3*Kt <= 192 fp32 columns, a ring of 2 to 4 accumulators), the epilogue warps read it with
 //     tcgen05.ld, apply the horizontal shifts with warp shuffles and write y directly in NCHW with
 //     128-byte coalesced rows.
 // Stride 2 (pad 1) keeps the even rows and columns of that stride-1 result: same operands, the
@@ -27,7 +27,8 @@
 // (group, filter tile, pixel tile), one CTA per SM walks it.
 //
 // Warp roles: warp 0 = TMA producer, warps 1 and 10 = single-thread MMA issuers for alternate tiles (warp 1 owns TMEM),
-// warps 2..9 = epilogue (TMEM lane quarter = warp_id % 4, two warps per quarter split the filters).  Every mbarrier wait is bounded: when a
+// warps 2..9 and 11..18 = two epilogue groups for alternate tiles (TMEM lane quarter = warp_id % 4).
+// Every mbarrier wait is bounded: when a
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
 // copies are waited for (bounded), TMEM is freed and the kernel returns.
 #include <cuda.h>
@@ -38,19 +39,20 @@ namespace gconv {
 
 namespace {
 
-constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each takes half of the filters
+constexpr int kEpiWarps = 8;             // warps of one epilogue group: two per TMEM lane quarter, each takes half of the filters
 constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the first is warp 1)
-constexpr int kThreads = 96 + 32 * kEpiWarps;
+constexpr int kEpi2First = kMmaWarp2 + 1;    // first warp of the second epilogue group
+constexpr int kThreads = 32 * (kEpi2First + kEpiWarps);
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 256;          // TMEM column offset between the two accumulator buffers
+constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 constexpr uint32_t kSpinLimit = 1u << 20;
 
 struct __align__(8) SharedCtl {
     unsigned long long full[8];
     unsigned long long empty[8];
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
-    unsigned long long xchg_bar[2];
+    unsigned long long tmem_full[kMaxAcc];
+    unsigned long long tmem_empty[kMaxAcc];
+    unsigned long long xchg_bar[kMaxAcc];
     unsigned long long b_full[2];   // resident weights of a (group, filter tile) have landed
     unsigned long long b_free[2];   // every MMA that read that weight buffer has completed
     uint32_t tmem_base;
@@ -151,7 +153,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                   const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
-    __shared__ float xchg[2][4][2][64];
+    __shared__ float xchg[kMaxAcc][4][2][64];
 
     if (packed[0] != tag) {
         if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
@@ -170,10 +172,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             mbar_init(smem_u32(&ctl.full[i]), 1);
             mbar_init(smem_u32(&ctl.empty[i]), 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kMaxAcc; ++i) {
             mbar_init(smem_u32(&ctl.tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl.tmem_empty[i]), kEpiWarps);
             mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl.b_full[i]), 1);
             mbar_init(smem_u32(&ctl.b_free[i]), 2);
         }
@@ -300,10 +304,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             uint32_t tcount = 0, switches = 0;
             int stage = 0;
             uint32_t ph = 0;
+            uint32_t buf = 0, bph = 0;      // accumulator ring position of the current tile and its pass parity
             int cur_gn = -1;
             uint32_t bres_addr = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x, ++tcount) {
+            for (int tile = blockIdx.x; tile < c.num_tiles && ok;
+                 tile += gridDim.x, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
                 uint32_t gn, mt;
                 c.div_mt.divmod((uint32_t)tile, gn, mt);
                 const bool mine = (tcount & 1) == mslot;
@@ -327,10 +333,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                     }
                     continue;
                 }
-                const uint32_t buf = tcount & 1;
-                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag, status, 200 + buf)) break;
+                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), bph ^ 1, abort_flag, status, 200 + buf)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)c.Np;
                 uint32_t acc = 0;
                 for (int ks = 0; ks < kstages; ++ks) {
                     if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 300 + stage)) { ok = false; break; }
@@ -360,15 +365,20 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
         }
     } else {
         // ---------------------------------------------------------------- epilogue warps
+        // Two groups of eight warps take alternate tiles, so one tile's TMEM reads, shuffles and stores overlap
+        // the next tile's.  With an even number of accumulators a buffer always belongs to the same group.
         const int wq = warp & 3;                       // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;              // which half of the tile's filters this warp stores
+        const uint32_t egroup = warp >= kEpi2First ? 1u : 0u;
+        const int half = ((warp - (egroup ? kEpi2First : 2)) >> 2);   // which half of the tile's filters this warp stores
         const int l = wq * 32 + lane;                  // pixel lane inside the tile
         const int Kt = c.Kt;
         const int kh = (Kt / 2 + 7) & ~7;              // filters of the first half (multiple of 8)
         const int kbeg = half == 0 ? 0 : kh;
         const int kend = half == 0 ? kh : Kt;
-        uint32_t tcount = 0;
-        for (int tile = blockIdx.x; tile < c.num_tiles; tile += gridDim.x, ++tcount) {
+        uint32_t buf = 0, bph = 0, tpar = 0;
+        for (int tile = blockIdx.x; tile < c.num_tiles;
+             tile += gridDim.x, tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
+            if (tpar != egroup) continue;              // the other group's tile
             uint32_t gn, mt;
             c.div_mt.divmod((uint32_t)tile, gn, mt);
             uint32_t n, i;
@@ -394,10 +404,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
             }
             const bool add_up = use_left && lane > 0;
             const bool add_dn = use_right && lane < 31;
-            const uint32_t buf = tcount & 1;
-            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), (tcount >> 1) & 1, abort_flag, status, 400 + buf)) break;
+            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), bph, abort_flag, status, 400 + buf)) break;
             tc_fence_after();
-            const uint32_t t0 = tmem_base + buf * kAccStride + ((uint32_t)(wq * 32) << 16);
+            const uint32_t t0 = tmem_base + buf * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
             // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
             float* yk = y + ((size_t)n * s.C_out + (size_t)gn * Kt + (size_t)kbeg) * OHW + fo;
             if (c.need_xchg) {
@@ -417,7 +426,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg_bar[buf]));
-                if (!mbar_wait_warp(smem_u32(&ctl.xchg_bar[buf]), (tcount >> 1) & 1, abort_flag, status, 500 + buf)) break;
+                if (!mbar_wait_warp(smem_u32(&ctl.xchg_bar[buf]), bph, abort_flag, status, 500 + buf)) break;
             }
             const bool edge_up = c.need_xchg && lane == 0 && wq > 0 && use_left;     // left neighbour is in the previous quarter
             const bool edge_dn = c.need_xchg && lane == 31 && wq < 3 && use_right;   // right neighbour is in the next quarter
@@ -573,6 +582,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
     }
+    c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.num_tiles = c.groups * c.NT * c.MT;
     c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)(c.seg_mode ? c.SPI : c.RB));
