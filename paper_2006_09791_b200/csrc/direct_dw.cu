@@ -1,0 +1,203 @@
+// DIRECT_TILED, depthwise kernel ("stream"): groups = C_in = C_out, 3x3, pad 1, stride 1 or 2, W % 4 == 0.
+//
+// Depthwise layers do 9 MACs per output and are bound by the HBM stream (2.25 FLOP per byte), so the
+// kernel is a software-pipelined stream: a thread owns a strip of 4 output columns of one plane and
+// walks down RH output rows.  Input rows arrive as aligned 16-byte loads that are issued one block of
+// rows ahead of their use (the next block's loads are in flight while the current block is computed),
+// the one-pixel left/right halos come from the neighbouring lanes by warp shuffle (a warp holds whole
+// rows: lane = strip-within-row, several rows' strips per warp), and every output row leaves as one
+// 16-byte store.  No shared memory, no barrier.  Sum order per output: (r, s) as in Algorithm 1.
+#include "gconv_internal.h"
+
+namespace gconv {
+
+namespace {
+
+constexpr int U = 4;   // output rows per pipeline block
+
+__device__ __forceinline__ float4 ldrow(const float* __restrict__ plane, int h, int H, int W, int col) {
+    if (h < 0 || h >= H) return make_float4(0.f, 0.f, 0.f, 0.f);
+    return __ldg(reinterpret_cast<const float4*>(plane + (size_t)h * W + col));
+}
+
+// ---- stride 1 -------------------------------------------------------------------------------------
+__device__ __forceinline__ void row_taps1(const float4 v, bool has_l, bool has_r, const float (&w)[3], float (&acc)[4]) {
+    float l = __shfl_up_sync(0xffffffffu, v.w, 1);
+    float r = __shfl_down_sync(0xffffffffu, v.x, 1);
+    l = has_l ? l : 0.f;
+    r = has_r ? r : 0.f;
+    acc[0] = fmaf(l, w[0], acc[0]);   acc[0] = fmaf(v.x, w[1], acc[0]); acc[0] = fmaf(v.y, w[2], acc[0]);
+    acc[1] = fmaf(v.x, w[0], acc[1]); acc[1] = fmaf(v.y, w[1], acc[1]); acc[1] = fmaf(v.z, w[2], acc[1]);
+    acc[2] = fmaf(v.y, w[0], acc[2]); acc[2] = fmaf(v.z, w[1], acc[2]); acc[2] = fmaf(v.w, w[2], acc[2]);
+    acc[3] = fmaf(v.z, w[0], acc[3]); acc[3] = fmaf(v.w, w[1], acc[3]); acc[3] = fmaf(r, w[2], acc[3]);
+}
+
+__global__ void __launch_bounds__(256)
+dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
+                    float* __restrict__ y, Status* status, uint32_t tag) {
+    const uint32_t tag_seen = __ldg(packed);
+    const float* __restrict__ wpk = reinterpret_cast<const float*>(packed + kHeaderBytes / 4);
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int sub = lane / c.XQ;                 // which of the warp's strips-of-rows this lane belongs to
+    const int xq = lane - sub * c.XQ;
+    // item = plane * chunks + chunk ; the warp holds `subs` consecutive items
+    const uint32_t item = warp_global * (uint32_t)c.subs + (uint32_t)sub;
+    const bool live = (sub < c.subs) && (item < c.items);
+    uint32_t plane_idx = 0, chunk = 0;
+    c.div_chunks.divmod(live ? item : 0u, plane_idx, chunk);
+    const int ch = (int)(plane_idx % (uint32_t)s.C_in);
+    const float* __restrict__ xp = x + (size_t)plane_idx * s.H * s.W;
+    float* __restrict__ yp = y + (size_t)plane_idx * s.H * s.W;
+    const int col = xq * 4;
+    const int p0 = (int)chunk * c.RH;
+    const int p1 = min(p0 + c.RH, s.H);
+    const bool has_l = xq > 0, has_r = xq < c.XQ - 1;
+    float w[3][3];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) w[i / 3][i % 3] = live ? __ldg(wpk + (size_t)ch * 9 + i) : 0.f;
+
+    // rows p-1 .. p+U of the current block; `live` only gates memory traffic, every lane runs the shuffles
+    float4 cur[U + 2], nxt[U];
+#pragma unroll
+    for (int j = 0; j < U + 2; ++j) cur[j] = live ? ldrow(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = p0; p < p0 + c.RH; p += U) {        // warp-uniform trip count
+#pragma unroll
+        for (int j = 0; j < U; ++j) {                  // next block's new rows, in flight during this block's math
+            const int h = p + U + 1 + j;
+            nxt[j] = (live && h <= p1) ? ldrow(xp, h, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            row_taps1(cur[j], has_l, has_r, w[0], acc);
+            row_taps1(cur[j + 1], has_l, has_r, w[1], acc);
+            row_taps1(cur[j + 2], has_l, has_r, w[2], acc);
+            if (live && p + j < p1 && tag_seen == tag)
+                *reinterpret_cast<float4*>(yp + (size_t)(p + j) * s.W + col) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        }
+        cur[0] = cur[U];
+        cur[1] = cur[U + 1];
+#pragma unroll
+        for (int j = 0; j < U; ++j) cur[2 + j] = nxt[j];
+    }
+    if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
+}
+
+// ---- stride 2 -------------------------------------------------------------------------------------
+// Four outputs q..q+3 read input columns 2q-1 .. 2q+7: two aligned float4 (a, b) and the previous lane's b.w.
+__device__ __forceinline__ void row_taps2(const float4 a, const float4 b, bool has_l, const float (&w)[3], float (&acc)[4]) {
+    float l = __shfl_up_sync(0xffffffffu, b.w, 1);
+    l = has_l ? l : 0.f;
+    acc[0] = fmaf(l, w[0], acc[0]);   acc[0] = fmaf(a.x, w[1], acc[0]); acc[0] = fmaf(a.y, w[2], acc[0]);
+    acc[1] = fmaf(a.y, w[0], acc[1]); acc[1] = fmaf(a.z, w[1], acc[1]); acc[1] = fmaf(a.w, w[2], acc[1]);
+    acc[2] = fmaf(a.w, w[0], acc[2]); acc[2] = fmaf(b.x, w[1], acc[2]); acc[2] = fmaf(b.y, w[2], acc[2]);
+    acc[3] = fmaf(b.y, w[0], acc[3]); acc[3] = fmaf(b.z, w[1], acc[3]); acc[3] = fmaf(b.w, w[2], acc[3]);
+}
+
+__global__ void __launch_bounds__(256)
+dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
+                    float* __restrict__ y, Status* status, uint32_t tag) {
+    const uint32_t tag_seen = __ldg(packed);
+    const float* __restrict__ wpk = reinterpret_cast<const float*>(packed + kHeaderBytes / 4);
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int sub = lane / c.XQ;
+    const int xq = lane - sub * c.XQ;
+    const uint32_t item = warp_global * (uint32_t)c.subs + (uint32_t)sub;
+    const bool live = (sub < c.subs) && (item < c.items);
+    uint32_t plane_idx = 0, chunk = 0;
+    c.div_chunks.divmod(live ? item : 0u, plane_idx, chunk);
+    const int ch = (int)(plane_idx % (uint32_t)s.C_in);
+    const float* __restrict__ xp = x + (size_t)plane_idx * s.H * s.W;
+    float* __restrict__ yp = y + (size_t)plane_idx * s.H_out * s.W_out;
+    const int col = xq * 8;                      // first of the 8 input columns of this strip
+    const int p0 = (int)chunk * c.RH;
+    const int p1 = min(p0 + c.RH, s.H_out);
+    const bool has_l = xq > 0;
+    const bool second_ok = col + 4 < s.W;        // W % 8 == 4: the last strip has only one vector
+    float w[3][3];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) w[i / 3][i % 3] = live ? __ldg(wpk + (size_t)ch * 9 + i) : 0.f;
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // input rows 2p-1, 2p, 2p+1 feed output row p; row 2p+1 is row 2(p+1)-1 of the next output
+    float4 ta = live ? ldrow(xp, 2 * p0 - 1, s.H, s.W, col) : z4;
+    float4 tb = (live && second_ok) ? ldrow(xp, 2 * p0 - 1, s.H, s.W, col + 4) : z4;
+    float4 ca[2], cb[2], na[2], nb[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        ca[j] = live ? ldrow(xp, 2 * p0 + j, s.H, s.W, col) : z4;
+        cb[j] = (live && second_ok) ? ldrow(xp, 2 * p0 + j, s.H, s.W, col + 4) : z4;
+    }
+    for (int p = p0; p < p0 + c.RH; ++p) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {                  // rows of the next output, in flight during this one's math
+            const int h = 2 * (p + 1) + j;
+            const bool need = live && (p + 1 < p1);
+            na[j] = need ? ldrow(xp, h, s.H, s.W, col) : z4;
+            nb[j] = (need && second_ok) ? ldrow(xp, h, s.H, s.W, col + 4) : z4;
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        row_taps2(ta, tb, has_l, w[0], acc);
+        row_taps2(ca[0], cb[0], has_l, w[1], acc);
+        row_taps2(ca[1], cb[1], has_l, w[2], acc);
+        if (live && p < p1 && tag_seen == tag) {
+            float* dst = yp + (size_t)p * s.W_out + xq * 4;
+            if ((s.W_out & 3) == 0) {
+                *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (xq * 4 + j < s.W_out) dst[j] = acc[j];
+            }
+        }
+        ta = ca[1];
+        tb = cb[1];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) { ca[j] = na[j]; cb[j] = nb[j]; }
+    }
+    if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
+}
+
+}  // namespace
+
+bool dw_supported(const Shape& s) {
+    if (!(s.KH == 3 && s.KW == 3 && s.dilation == 1 && s.pad == 1 && (s.stride == 1 || s.stride == 2))) return false;
+    if (!(s.Cg == 1 && s.Kg == 1)) return false;
+    if (s.W % 4 != 0) return false;
+    const int xq = s.stride == 1 ? s.W / 4 : (s.W + 7) / 8;
+    if (xq > 32) return false;
+    return (unsigned long long)s.N * s.C_in * s.H_out < (1ull << 30);
+}
+
+DwCfg dw_config(const Shape& s, int sm_count) {
+    DwCfg c;
+    c.XQ = s.stride == 1 ? s.W / 4 : (s.W + 7) / 8;
+    c.subs = 32 / c.XQ;
+    // rows per thread: long strips amortise the two halo rows, short ones give more parallelism; aim for
+    // at least ~6 waves of 1024 threads per SM
+    const long long planes = (long long)s.N * s.C_in;
+    int rh = s.H_out;
+    while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < 6LL * 1024 * sm_count) rh = (rh + 1) / 2;
+    rh = ((rh + U - 1) / U) * U;
+    c.RH = rh;
+    c.chunks = (s.H_out + rh - 1) / rh;
+    c.div_chunks = make_fastdiv((uint32_t)c.chunks);
+    c.items = (uint32_t)(planes * c.chunks);
+    const uint32_t warps = (c.items + c.subs - 1) / c.subs;
+    c.blocks = (warps + 7) / 8;
+    return c;
+}
+
+cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
+                       cudaStream_t st) {
+    const DwCfg c = dw_config(s, sm_count);
+    const uint32_t tag = pack_tag(s, GCONV_VARIANT_DIRECT_TILED);
+    if (s.stride == 1)
+        dw_stream_s1_kernel<<<c.blocks, 256, 0, st>>>(s, c, x, reinterpret_cast<const uint32_t*>(packed), y, status, tag);
+    else
+        dw_stream_s2_kernel<<<c.blocks, 256, 0, st>>>(s, c, x, reinterpret_cast<const uint32_t*>(packed), y, status, tag);
+    return cudaGetLastError();
+}
+
+}  // namespace gconv

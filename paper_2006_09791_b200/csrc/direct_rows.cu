@@ -69,13 +69,12 @@ __device__ __forceinline__ void load_row(const float* __restrict__ row, bool row
 }
 
 template <int S, int KT, int PR, bool VEC>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, (KT <= 2 && VEC) ? 8 : 1)
 direct_rows_kernel(const Shape s, const RowsCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                    float* __restrict__ y, Status* status, uint32_t tag) {
-    if (packed[0] != tag) {
-        if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
-        return;
-    }
+    // The header tag is loaded now but only examined right before the stores, so the check costs no
+    // memory round trip ahead of the input loads; a mismatch still leaves y untouched.
+    const uint32_t tag_seen = __ldg(packed);
     const float* __restrict__ wpk = reinterpret_cast<const float*>(packed + kHeaderBytes / 4);
     const uint32_t item = blockIdx.x * blockDim.x + threadIdx.x;
     if (item >= c.items) return;
@@ -140,6 +139,10 @@ direct_rows_kernel(const Shape s, const RowsCfg c, const float* __restrict__ x, 
         }
     }
 
+    if (tag_seen != tag) {
+        if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
+        return;
+    }
     const size_t oplane = (size_t)s.H_out * s.W_out;
     float* yb = y + ((size_t)n * s.C_out + (size_t)g * KT) * oplane;
     const bool vec_store = ((s.W_out & 3) == 0);

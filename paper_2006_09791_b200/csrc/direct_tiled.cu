@@ -280,6 +280,7 @@ static cudaError_t launch_tiled(const Shape& s, const TiledCfg& c, const float* 
 
 cudaError_t tiled_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
                           cudaStream_t st) {
+    if (dw_supported(s)) return dw_forward(s, x, packed, y, status, sm_count, st);
     if (rows_supported(s)) return rows_forward(s, x, packed, y, status, st);
     const TiledCfg c = tiled_config(s, sm_count);
 #define GCONV_TILED_CASE(S, K) \

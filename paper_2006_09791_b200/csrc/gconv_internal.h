@@ -78,6 +78,17 @@ bool rows_supported(const Shape& s);
 RowsCfg rows_config(const Shape& s);
 cudaError_t rows_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, cudaStream_t st);
 
+// DIRECT_TILED, depthwise stream kernel: a warp holds `subs` row strips of XQ lanes each.
+struct DwCfg {
+    int XQ, subs, RH, chunks;   // lanes per row, rows' strips per warp, output rows per thread, row chunks per plane
+    FastDiv div_chunks;
+    uint32_t items, blocks;
+};
+bool dw_supported(const Shape& s);
+DwCfg dw_config(const Shape& s, int sm_count);
+cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
+                       cudaStream_t st);
+
 // DIRECT_TILED: launch geometry chosen on the host from the shape.
 struct TiledCfg {
     int TXT, TY, KQ, GB, KT, CCH;          // x threads, rows, filter slabs, groups per CTA, filters per thread, channel chunk
