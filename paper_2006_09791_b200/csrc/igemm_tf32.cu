@@ -108,6 +108,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -149,7 +155,8 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
 
 
 __global__ void __launch_bounds__(kThreads, 1)
-igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const IgemmCfg c,
+igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xmap4, const Shape s,
+                  const IgemmCfg c,
                   const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
@@ -216,7 +223,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
         uint32_t ph = 0;                                   // phase parity of the current pass over the stage ring
         int cur_gn = -1;
         bool ok = true;
-        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
+            if (c.fast4) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap4) : "memory");
+        }
         for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
             uint32_t gn, mt;
             c.div_mt.divmod((uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
@@ -254,6 +264,24 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                 my_f = (int)i * c.R * s.W + 32 * (lane & 3);
             }
             const bool issuer = lane < c.nseg;
+            // One 4-D box (32 pixels x CK channels x nseg segments) replaces the per-segment copies whenever the
+            // tile's segments are one contiguous run that stays inside the image plane for the tap at hand; the
+            // plane's first and last tiles (whose halo is out of range and must be zero-filled) keep the
+            // per-segment copies, where out-of-range means out of the plane.
+            int tile_n = 0, tile_f0 = 0;
+            bool contiguous = false;
+            if (c.fast4) {
+                uint32_t n, i;
+                if (c.seg_mode) {
+                    c.div_spi.divmod(mt * 4u, n, i);
+                    tile_f0 = (int)i * 32;
+                } else {
+                    c.div_spi.divmod(mt, n, i);
+                    tile_f0 = (int)i * c.R * s.W;
+                }
+                tile_n = (int)n;
+                contiguous = true;
+            }
             int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
                 if (!mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
@@ -265,8 +293,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const Shape s, const
                     if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
                 }
                 __syncwarp();
-                if (issuer)
+                const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
+                if (contiguous && lo >= 0 && lo + c.nseg * 32 <= HW) {
+                    if (lane == 0) tma_load_4d(a_dst, &xmap4, lo, g * c.Cg + ch * c.CK, 0, tile_n, full);
+                } else if (issuer) {
                     tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, g * c.Cg + ch * c.CK, my_n, full);
+                }
                 if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
@@ -582,6 +614,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
     }
+    c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.num_tiles = c.groups * c.NT * c.MT;
     c.div_mt = make_fastdiv((uint32_t)c.MT);
@@ -632,6 +665,23 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    // 4-D view for whole-tile copies: (pixel, channel, 32-pixel segment, image); the segment axis re-walks the
+    // pixel axis in steps of 128 bytes, so one box covers nseg consecutive segments.
+    IgemmCfg cfg = c;
+    CUtensorMap xmap4 = xmap;
+    cfg.fast4 = 0;
+    if (c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
+        const cuuint64_t dims4[4] = {HW, (cuuint64_t)s.C_in, 8, (cuuint64_t)s.N};
+        const cuuint64_t strides4[3] = {HW * 4, 128, HW * 4 * (cuuint64_t)s.C_in};
+        const cuuint32_t box4[4] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.nseg, 1};
+        const cuuint32_t estr4[4] = {1, 1, 1, 1};
+        if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims4, strides4, box4, estr4,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+            cfg.fast4 = 1;
+        else
+            xmap4 = xmap;
+    }
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -640,7 +690,7 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    igemm_tf32_kernel<<<c.grid, kThreads, c.smem_bytes, st>>>(xmap, s, c, reinterpret_cast<const uint32_t*>(packed), y, status,
+    igemm_tf32_kernel<<<c.grid, kThreads, c.smem_bytes, st>>>(xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
                                                               pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
     return cudaGetLastError();
 }
