@@ -117,7 +117,8 @@ struct IgemmCfg {
     int seg_fstep;           // flat-pixel step between consecutive segments of an image
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int nacc;                // accumulator buffers in the TMEM ring
-    int fast4;               // a 4-D tensor map for whole-tile copies is available
+    int fast4;               // a second tensor map for whole-tile copies is available
+    int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)
     int num_tiles, stages, grid;
     FastDiv div_nt;                   // (group, filter tile) index -> group
     FastDiv div_mt, div_spi, div_w;   // tile -> (group/filter tile, pixel tile); pixel tile -> (image, segment or row block); pixel -> (row, column)

@@ -114,6 +114,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -268,9 +275,14 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             // tile's segments are one contiguous run that stays inside the image plane for the tap at hand; the
             // plane's first and last tiles (whose halo is out of range and must be zero-filled) keep the
             // per-segment copies, where out-of-range means out of the plane.
-            int tile_n = 0, tile_f0 = 0;
+            int tile_n = 0, tile_f0 = 0, rb_p0 = 0;
             bool contiguous = false;
-            if (c.fast4) {
+            if (c.rowbox) {
+                uint32_t n, i;
+                c.div_spi.divmod(mt, n, i);
+                tile_n = (int)n;
+                rb_p0 = (int)i * c.R;                     // first output row of the tile
+            } else if (c.fast4) {
                 uint32_t n, i;
                 if (c.seg_mode) {
                     c.div_spi.divmod(mt * 4u, n, i);
@@ -294,7 +306,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 }
                 __syncwarp();
                 const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
-                if (contiguous && lo >= 0 && lo + c.nseg * 32 <= HW) {
+                if (c.rowbox) {
+                    // one 5-D box: 32 pixels x CK channels x SR row segments x (RT + 2) rows; rows outside the image and
+                    // columns past W are zero-filled by TMA, which is exactly the padding
+                    if (lane == 0) tma_load_5d(a_dst, &xmap4, 0, g * c.Cg + ch * c.CK, 0, rb_p0 - 1, tile_n, full);
+                } else if (contiguous && lo >= 0 && lo + c.nseg * 32 <= HW) {
                     if (lane == 0) tma_load_4d(a_dst, &xmap4, lo, g * c.Cg + ch * c.CK, 0, tile_n, full);
                 } else if (issuer) {
                     tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, g * c.Cg + ch * c.CK, my_n, full);
@@ -416,7 +432,17 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             uint32_t n, i;
             int f;
             bool valid;
-            if (c.seg_mode) {
+            if (c.rowbox) {
+                // quarter wq is segment h = wq % SR of row p0 + wq / SR; the last segment of a two-segment row is
+                // shifted left to end at column W, and each column is stored by the segment that holds both of its
+                // horizontal neighbours
+                c.div_spi.divmod(mt, n, i);
+                const int h = c.SR == 2 ? (wq & 1) : 0;
+                const int row = (int)i * c.R + (c.SR == 2 ? (wq >> 1) : wq);
+                const int col = (h ? s.W - 32 : 0) + lane;
+                valid = row < s.H && col < s.W && (c.SR == 1 || (h == 0 ? col <= 30 : col >= 31));
+                f = row * s.W + (col < s.W ? col : s.W - 1);
+            } else if (c.seg_mode) {
                 c.div_spi.divmod(mt * 4u + (uint32_t)wq, n, i);
                 f = (int)i * c.seg_fstep + lane;
                 valid = (int)n < s.N;
@@ -604,12 +630,35 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) {
         c.MT = s.N * c.RB;
         c.need_xchg = 1;
     }
+    // Row boxes: for widths that do not divide 32 a tile can instead be RT whole rows of SR 32-pixel segments each
+    // (the second segment of a row shifted left to end at column W).  Every vertical tap is then a whole number of
+    // segments away, so one staged block (tile + a row above and below, one 5-D TMA box) serves all three taps, and
+    // each segment contains the horizontal neighbours of the columns it stores (no exchange between warps).  Used
+    // when it wastes at most a quarter more lanes than the flat tiling.
+    c.rowbox = 0;
+    c.SR = 0;
+    if (!c.seg_mode && s.W <= 62) {
+        const int sr = s.W <= 32 ? 1 : 2;
+        const double util_box = (double)s.W / (32.0 * sr), util_flat = (double)((128 / s.W) * s.W) / 128.0;
+        if (util_box >= 0.8 * util_flat) {
+            c.rowbox = 1;
+            c.SR = sr;
+            c.R = 4 / sr;                                // rows per tile
+            c.RB = (s.H + c.R - 1) / c.R;
+            c.MT = s.N * c.RB;
+            c.need_xchg = 0;
+        }
+    }
     // Row halo: when a row is a whole number of 32-pixel segments the three vertical taps are views of
     // one staged block (tile + one row above and below), so the input crosses L2 -> shared memory once.
     c.nr = 1;
     c.nseg = 4;
     c.wseg = 0;
-    if (s.stride == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
+    if (c.rowbox) {
+        c.nr = 3;
+        c.wseg = c.SR;
+        c.nseg = 4 + 2 * c.SR;
+    } else if (s.stride == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
         c.nr = 3;
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
@@ -670,7 +719,19 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
     IgemmCfg cfg = c;
     CUtensorMap xmap4 = xmap;
     cfg.fast4 = 0;
-    if (c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
+    if (c.rowbox) {
+        // (column, channel, row segment, row, image); the segment axis steps (W - 32) columns
+        const cuuint64_t dims5[5] = {(cuuint64_t)s.W, (cuuint64_t)s.C_in, (cuuint64_t)c.SR, (cuuint64_t)s.H, (cuuint64_t)s.N};
+        const cuuint64_t strides5[4] = {HW * 4, c.SR == 2 ? (cuuint64_t)(s.W - 32) * 4 : 128, (cuuint64_t)s.W * 4,
+                                        HW * 4 * (cuuint64_t)s.C_in};
+        const cuuint32_t box5[5] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.SR, (cuuint32_t)(c.R + 2), 1};
+        const cuuint32_t estr5[5] = {1, 1, 1, 1, 1};
+        if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float*>(x), dims5, strides5, box5, estr5,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+        cfg.fast4 = 1;   // the second map is in use (prefetch it)
+    } else if (c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
         const cuuint64_t dims4[4] = {HW, (cuuint64_t)s.C_in, 8, (cuuint64_t)s.N};
         const cuuint64_t strides4[3] = {HW * 4, 128, HW * 4 * (cuuint64_t)s.C_in};
         const cuuint32_t box4[4] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.nseg, 1};
