@@ -169,10 +169,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     __shared__ SharedCtl ctl;
     __shared__ float xchg[kMaxAcc][4][2][64];
 
-    if (packed[0] != tag) {
-        if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
-        return;
-    }
+    // Programmatic dependent launch: let the next kernel in the stream be scheduled as SMs free up, and run this
+    // kernel's own set-up (barriers, TMEM) while the previous kernel drains; nothing below touches global memory
+    // until griddepcontrol.wait has returned, i.e. until the previous kernel's writes are complete and visible.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint8_t* __restrict__ wblocks = reinterpret_cast<const uint8_t*>(packed) + kHeaderBytes;
 
     const int warp = threadIdx.x >> 5;
@@ -208,6 +208,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool tag_ok = (packed[0] == tag);   // uniform across the CTA
+    if (!tag_ok && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 
     // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
     // segments of one vertical tap (nr = 1, stages run chunk-major, tap-minor), or the tile plus its
@@ -222,7 +225,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     const int HW = s.H * s.W;
     const size_t OHW = (size_t)s.H_out * s.W_out;
 
-    if (warp == 0) {
+    if (!tag_ok) {
+        // wrong weights: no role runs, y stays untouched; fall through to the common exit (TMEM is freed there)
+    } else if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
         uint32_t it = 0, switches = 0;
@@ -751,9 +756,18 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    igemm_tf32_kernel<<<c.grid, kThreads, c.smem_bytes, st>>>(xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
-                                                              pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
-    return cudaGetLastError();
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)c.grid);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = c.smem_bytes;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, igemm_tf32_kernel, xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
+                              pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
 }
 
 
