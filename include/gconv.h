@@ -119,6 +119,10 @@ int gconv_pack_weights(gconv_desc_t desc, const float *w_ochw, void *w_packed, v
  *   x_nchw    device, fp32 [N, C_in, H, W], read only; must not overlap y.
  *   w_packed  device, produced by gconv_pack_weights on a descriptor of the same shape and variant.
  *   y_nchw    device, fp32 [N, C_out, H_out, W_out], every element written.
+ * For layers whose width is not a multiple of 4 the tensor-core variant computes on a zero-padded copy of x that
+ * it keeps in a device scratch buffer owned by the descriptor: that buffer is allocated (cudaMalloc) by the first
+ * gconv_forward of such a descriptor -- make that call outside any stream capture -- and freed by
+ * gconv_desc_destroy; two concurrent forwards of ONE such descriptor would race on it.
  * Kernel launches only, on `stream`; deterministic (no atomics on y).  A w_packed made for another shape or
  * variant is detected on the device: y is left unwritten and gconv_last_status reports
  * GCONV_ERR_PACK_MISMATCH.  Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_CUDA.
@@ -159,7 +163,9 @@ int gconv_forward_host(gconv_desc_t desc, const float *x_host, const void *w_pac
  * All calls share the one array, which still holds the previous call's data: the status block is
  * cleared and the staging regions are rewritten on every call, so results never depend on it, but
  * calls that overlap on the GPU (two streams, two threads) race and must be serialised by the caller.
- * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT (w_packed), GCONV_ERR_TOO_LARGE, GCONV_ERR_CUDA.
+ * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT (w_packed), GCONV_ERR_TOO_LARGE, GCONV_ERR_CUDA, and
+ * GCONV_ERR_UNSUPPORTED for the layers that need the padded-copy scratch described at gconv_forward
+ * (tensor-core variant, width not a multiple of 4): force another variant for those.
  */
 int gconv_forward_host_static(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host, void *stream);
 

@@ -44,6 +44,8 @@ extern "C" int gconv_forward_host_static(gconv_desc_t d, const float* x_host, co
     const size_t xb = sizeof(float) * (size_t)s.N * s.C_in * s.H * s.W;
     const size_t yb = sizeof(float) * (size_t)s.N * s.C_out * s.H_out * s.W_out;
     if (round256(xb) + round256(yb) > kStageBytes) return GCONV_ERR_TOO_LARGE;
+    // layers that the tensor-core variant runs on a padded copy of x need a second scratch buffer: not offered here
+    if (d->variant == GCONV_VARIANT_IGEMM_TF32 && igemm_scratch_bytes(s) > 0) return GCONV_ERR_UNSUPPORTED;
 
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -75,7 +77,7 @@ extern "C" int gconv_forward_host_static(gconv_desc_t d, const float* x_host, co
     if (e == cudaSuccess) {
         switch (d->variant) {
             case GCONV_VARIANT_IGEMM_TF32:
-                e = igemm_forward(s, x_stage, w_packed, y_stage, status, g_sm_count[dev], st);
+                e = igemm_forward(s, x_stage, w_packed, y_stage, status, g_sm_count[dev], st, nullptr);
                 break;
             case GCONV_VARIANT_DIRECT_TILED:
                 e = tiled_forward(s, x_stage, w_packed, y_stage, status, g_sm_count[dev], st);

@@ -43,6 +43,11 @@ int ensure_device_state(gconv_desc* d) {
         cudaFree(d->status_dev);
         d->status_dev = nullptr;
     }
+    if (d->scratch != nullptr) {
+        cudaFree(d->scratch);
+        d->scratch = nullptr;
+        d->scratch_bytes = 0;
+    }
     e = cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return fail_cuda(d, e);
     e = cudaMalloc(&d->status_dev, sizeof(Status));
@@ -89,6 +94,8 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
     d->device = -1;
     d->sm_count = 0;
     d->last_cuda_error = 0;
+    d->scratch = nullptr;
+    d->scratch_bytes = 0;
     *out = d;
     return GCONV_OK;
 }
@@ -96,6 +103,7 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
 int gconv_desc_destroy(gconv_desc_t d) {
     if (d == nullptr) return GCONV_OK;
     if (d->status_dev != nullptr) cudaFree(d->status_dev);
+    if (d->scratch != nullptr) cudaFree(d->scratch);
     delete d;
     return GCONV_OK;
 }
@@ -180,9 +188,19 @@ int gconv_forward(gconv_desc_t d, const float* x, const void* w_packed, float* y
         case GCONV_VARIANT_DIRECT_TILED:
             e = tiled_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
             break;
-        case GCONV_VARIANT_IGEMM_TF32:
-            e = igemm_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
+        case GCONV_VARIANT_IGEMM_TF32: {
+            const size_t need = igemm_scratch_bytes(d->s);
+            if (need > d->scratch_bytes) {   // first forward of a layer that runs on a padded copy of x
+                if (d->scratch != nullptr) cudaFree(d->scratch);
+                d->scratch = nullptr;
+                d->scratch_bytes = 0;
+                e = cudaMalloc(&d->scratch, need);
+                if (e != cudaSuccess) return fail_cuda(d, e);
+                d->scratch_bytes = need;
+            }
+            e = igemm_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st, d->scratch);
             break;
+        }
         case GCONV_VARIANT_DIRECT_GENERIC:
         default:
             e = generic_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st);
@@ -208,7 +226,10 @@ int gconv_forward_host(gconv_desc_t d, const float* x_host, const void* w_packed
     return GCONV_OK;
 }
 
-int gconv_forward_launches(gconv_desc_t d) { return d == nullptr ? 0 : 1; }
+int gconv_forward_launches(gconv_desc_t d) {
+    if (d == nullptr) return 0;
+    return (d->variant == GCONV_VARIANT_IGEMM_TF32 && igemm_scratch_bytes(d->s) > 0) ? 2 : 1;
+}
 
 int gconv_last_status(gconv_desc_t d, void* stream) {
     if (d == nullptr) return GCONV_ERR_NULL;

@@ -23,6 +23,8 @@ struct gconv_desc {
     int device;                  // device the status block lives on (-1 = none yet)
     int sm_count;
     int last_cuda_error;
+    float* scratch;              // lazily allocated device scratch (padded input copy), nullptr for most shapes
+    size_t scratch_bytes;
 };
 
 namespace gconv {
@@ -118,6 +120,7 @@ struct IgemmCfg {
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int nacc;                // accumulator buffers in the TMEM ring
     int fast4;               // a second tensor map for whole-tile copies is available
+    int padded, Hv, Wv;      // the kernel computes on a zero-padded copy of x; valid extent of the plane
     int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)
     int num_tiles, stages, grid;
     FastDiv div_nt;                   // (group, filter tile) index -> group
@@ -129,7 +132,8 @@ bool igemm_supported(const Shape& s);
 IgemmCfg igemm_config(const Shape& s, int sm_count);
 size_t igemm_packed_bytes(const Shape& s);
 cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_t st);
+size_t igemm_scratch_bytes(const Shape& s);   // device scratch the forward needs (padded copy of x), 0 for most shapes
 cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
-                          cudaStream_t st);
+                          cudaStream_t st, float* scratch);
 
 }  // namespace gconv

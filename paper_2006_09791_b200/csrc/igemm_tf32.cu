@@ -460,7 +460,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             c.div_w.divmod((uint32_t)f, prow, q);
             const bool use_left = q > 0;
             const bool use_right = (int)q < s.W - 1;
-            int fo = f;                                  // position in the output plane
+            // s.H x s.W is the (possibly padded) plane the kernel computes on; only the first Hv x Wv pixels exist in y
+            valid = valid && (int)prow < c.Hv && (int)q < c.Wv;
+            int fo = (int)prow * s.W_out + (int)q;       // position in the output plane
             if (s.stride == 2) {                         // stride 2 keeps the even rows and columns of the stride-1 result
                 valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
                 fo = (int)(prow >> 1) * s.W_out + (int)(q >> 1);
@@ -586,6 +588,44 @@ EncodeTiledFn get_encode_fn() {
 
 }  // namespace
 
+// Widths that are not a multiple of 4 cannot be addressed by TMA (row shifts must be 16-byte aligned), so such
+// layers run on a zero-padded copy of x: rows padded to a multiple of 4 columns (and, when that width divides 32,
+// the row count padded until the plane is a whole number of 32-pixel segments).  The zero columns and rows are
+// exactly the convolution's right and bottom padding; outputs that fall in them are never stored.
+struct IgemmGeom {
+    int Hp, Wp;
+    bool padded;
+};
+static IgemmGeom igemm_geom(const Shape& s) {
+    IgemmGeom g;
+    g.Wp = (s.W + 3) & ~3;
+    g.Hp = s.H;
+    g.padded = g.Wp != s.W;
+    if (g.padded && 32 % g.Wp == 0)
+        while ((g.Hp * g.Wp) % 32 != 0) ++g.Hp;
+    return g;
+}
+
+namespace {
+__global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict__ xp, size_t planes, int H, int W, int Hp, int Wp) {
+    const size_t per_plane = (size_t)Hp * (Wp / 4);
+    const size_t total = planes * per_plane;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t plane = i / per_plane;
+        const int rem = (int)(i - plane * per_plane);
+        const int h = rem / (Wp / 4), w4 = (rem - h * (Wp / 4)) * 4;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (h < H) {
+            const float* src = x + (plane * H + h) * (size_t)W;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (w4 + j < W) v[j] = __ldg(src + w4 + j);
+        }
+        *reinterpret_cast<float4*>(xp + (plane * Hp + h) * (size_t)Wp + w4) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+}  // namespace
+
 static int igemm_merge(const Shape& s) {
     int m = 1;
     while (m * 2 <= s.groups && s.groups % (m * 2) == 0 && s.Cg * m * 2 <= 32 && s.Kg * m * 2 <= 64) m *= 2;
@@ -596,14 +636,27 @@ bool igemm_supported(const Shape& s) {
     if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.pad == 1 && s.dilation == 1)) return false;
     const int m = igemm_merge(s);
     if ((s.Cg * m) % 8 != 0 || (s.Kg * m) % 8 != 0) return false;
-    if (s.W % 4 != 0 || s.W > 128) return false;
-    if ((long long)s.H * s.W < 32) return false;
+    const IgemmGeom ge = igemm_geom(s);
+    if (ge.Wp > 128) return false;
+    if ((long long)ge.Hp * ge.Wp < 32) return false;
     if (s.C_in > 65535 * 8) return false;
     return true;
 }
 
-IgemmCfg igemm_config(const Shape& s, int sm_count) {
+size_t igemm_scratch_bytes(const Shape& s) {
+    const IgemmGeom ge = igemm_geom(s);
+    return ge.padded ? sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp : 0;
+}
+
+IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     IgemmCfg c;
+    const IgemmGeom ge = igemm_geom(s_true);
+    Shape s = s_true;          // the plane the kernel computes on
+    s.H = ge.Hp;
+    s.W = ge.Wp;
+    c.Hv = s_true.H;
+    c.Wv = s_true.W;
+    c.padded = ge.padded ? 1 : 0;
     c.merge = igemm_merge(s);
     c.groups = s.groups / c.merge;
     c.Cg = s.Cg * c.merge;
@@ -704,9 +757,24 @@ cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_
     return cudaGetLastError();
 }
 
-cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
-                          cudaStream_t st) {
-    const IgemmCfg c = igemm_config(s, sm_count);
+cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* packed, float* y, Status* status, int sm_count,
+                          cudaStream_t st, float* scratch) {
+    const IgemmCfg c = igemm_config(s_true, sm_count);
+    Shape s = s_true;
+    const float* x = x_in;
+    if (c.padded) {
+        if (scratch == nullptr) return cudaErrorInvalidValue;
+        const IgemmGeom ge = igemm_geom(s_true);
+        const size_t planes = (size_t)s.N * s.C_in;
+        const size_t total = planes * ge.Hp * (ge.Wp / 4);
+        const int blocks = (int)((total + 255) / 256 < (size_t)sm_count * 16 ? (total + 255) / 256 : (size_t)sm_count * 16);
+        igemm_pad_kernel<<<blocks, 256, 0, st>>>(x_in, scratch, planes, s.H, s.W, ge.Hp, ge.Wp);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        s.H = ge.Hp;
+        s.W = ge.Wp;
+        x = scratch;
+    }
     EncodeTiledFn encode = get_encode_fn();
     if (encode == nullptr) return cudaErrorNotSupported;
     CUtensorMap xmap;
@@ -767,7 +835,7 @@ cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, fl
     lc.attrs = attr;
     lc.numAttrs = 1;
     return cudaLaunchKernelEx(&lc, igemm_tf32_kernel, xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
-                              pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
+                              pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32));
 }
 
 

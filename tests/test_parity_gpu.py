@@ -66,6 +66,8 @@ ODD_SHAPES = [
     (1, 64, 9, 64, 64, 3, 3, 2, 1, 1, 4), (2, 96, 10, 8, 96, 3, 3, 1, 1, 1, 1), (1, 128, 6, 128, 128, 3, 3, 1, 1, 1, 2),
     (2, 12, 13, 12, 12, 3, 3, 2, 1, 1, 12), (1, 8, 9, 128, 8, 3, 3, 1, 1, 1, 8), (3, 20, 57, 56, 20, 3, 3, 1, 1, 1, 20),
     (2, 6, 30, 28, 6, 3, 3, 2, 1, 1, 6), (1, 40, 5, 4, 40, 3, 3, 1, 1, 1, 40), (2, 7, 3, 8, 7, 3, 3, 2, 1, 1, 7),
+    (3, 16, 14, 14, 32, 3, 3, 2, 1, 1, 2), (2, 8, 7, 7, 8, 3, 3, 1, 1, 1, 1), (1, 32, 9, 30, 32, 3, 3, 1, 1, 1, 4),
+    (2, 24, 5, 6, 24, 3, 3, 1, 1, 1, 3), (1, 16, 21, 50, 16, 3, 3, 2, 1, 1, 2), (2, 8, 3, 126, 8, 3, 3, 1, 1, 1, 1),
     (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
 ]
 
