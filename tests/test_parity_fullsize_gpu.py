@@ -1,0 +1,84 @@
+"""GPU parity at the benchmark's full sizes.  The whole tensor is computed on the GPU (selector's variant,
+same launch path as bench.py, including a CUDA-graph replay) and compared with the oracle on sampled
+(image, group) slices: for a sampled pair the oracle convolves x[n, group's channels] with the group's
+filters (a groups = 1 problem it finishes in well under a second) and every element of y[n, group's
+filters] must agree within the variant's tolerance, scaled by the largest reference magnitude seen."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2006_09791_b200 import build as gbuild
+from paper_2006_09791_b200 import gconv, synth
+from paper_2006_09791_b200.workloads import sweep_layers, wrn_stack
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gbuild.build()
+
+
+def _run_full(L, x, w, use_graph):
+    dev = torch.device("cuda:0")
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            xd = torch.from_numpy(x).to(dev)
+            wd = torch.from_numpy(w).to(dev)
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            y = torch.full((L.y_elems,), float("nan"), dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(d, wd, wp, s)
+            gconv.gconv_forward(d, xd, wp, y, s)          # also allocates whatever the descriptor needs
+            if use_graph:
+                s.synchronize()
+                y.fill_(float("nan"))
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=s):
+                    gconv.gconv_forward(d, xd, wp, y, s)
+                graph.replay()
+            s.synchronize()
+        assert gconv.gconv_last_status(d, s) == gconv.GCONV_OK
+        return y.cpu().numpy().reshape(L.N, L.C_out, L.H_out, L.W_out), gconv.gconv_variant(d)
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def _check_samples(L, y, x, w, variant, samples):
+    tol = gconv.VARIANT_TOLERANCE[variant]
+    assert np.all(np.isfinite(y)), "non-finite output (an element was never written?)"
+    refs, errs = [], []
+    for n, g in samples:
+        xs = x[n:n + 1, g * L.Cg:(g + 1) * L.Cg]
+        ws = w[g * L.Kg:(g + 1) * L.Kg]
+        ref = oracle.gconv_ref(xs, ws, L.stride, L.pad, L.dilation, 1, threads=16)[0]
+        refs.append(np.max(np.abs(ref)))
+        errs.append(np.max(np.abs(y[n, g * L.Kg:(g + 1) * L.Kg].astype(np.float64) - ref)))
+    rel = max(errs) / max(refs)
+    assert rel <= tol, "%s groups=%d variant %s: sampled rel err %.3e > %.1e" % (L.name, L.groups, gconv.variant_name(variant), rel, tol)
+
+
+def _samples(L, k, seed):
+    rng = np.random.RandomState(seed)
+    out = {(0, 0), (L.N - 1, L.groups - 1)}           # first and last slices always
+    while len(out) < k:
+        out.add((int(rng.randint(L.N)), int(rng.randint(L.groups))))
+    return sorted(out)
+
+
+@pytest.mark.parametrize("groups", [1, 4, 16])
+def test_wrn_stack_at_batch_128(groups):
+    for i, L in enumerate(wrn_stack(groups, 128)):
+        x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, synth.layer_seed(77, i, groups), L.x_dist)
+        y, v = _run_full(L, x, w, use_graph=(i % 2 == 0))
+        _check_samples(L, y, x, w, v, _samples(L, 6, i))
+
+
+@pytest.mark.parametrize("idx", [0, 3, 6, 8])     # groups 1, 8, 64, 256 of the sweep to depthwise
+def test_group_sweep_at_batch_32(idx):
+    L = sweep_layers(32)[idx]
+    x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(78, idx), L.x_dist)
+    y, v = _run_full(L, x, w, use_graph=True)
+    _check_samples(L, y, x, w, v, _samples(L, 3 if L.groups == 1 else 6, idx))
