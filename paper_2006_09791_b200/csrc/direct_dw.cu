@@ -1,8 +1,9 @@
-// DIRECT_TILED, depthwise kernel ("stream"): groups = C_in = C_out, 3x3, pad 1, stride 1 or 2, W % 4 == 0.
+// DIRECT_TILED, depthwise kernel ("stream"): groups = C_in = C_out, 3x3, pad 1, stride 1 or 2, W <= 128 (256 for stride 2).
 //
 // Depthwise layers do 9 MACs per output and are bound by the HBM stream (2.25 FLOP per byte), so the
 // kernel is a software-pipelined stream: a thread owns a strip of 4 output columns of one plane and
-// walks down RH output rows.  Input rows arrive as aligned 16-byte loads that are issued one block of
+// walks down RH output rows.  Input rows arrive as aligned 16-byte loads (four scalar loads when W is not a
+// multiple of 4) that are issued one block of
 // rows ahead of their use (the next block's loads are in flight while the current block is computed),
 // the one-pixel left/right halos come from the neighbouring lanes by warp shuffle (a warp holds whole
 // rows: lane = strip-within-row, several rows' strips per warp), and every output row leaves as one
@@ -15,9 +16,32 @@ namespace {
 
 constexpr int U = 4;   // output rows per pipeline block
 
+// Four consecutive pixels of row h starting at column col (zero outside the image).  VEC: W % 4 == 0, so the
+// address is 16-byte aligned and the four pixels are in range; otherwise four bounds-checked scalar loads.
+template <bool VEC>
 __device__ __forceinline__ float4 ldrow(const float* __restrict__ plane, int h, int H, int W, int col) {
     if (h < 0 || h >= H) return make_float4(0.f, 0.f, 0.f, 0.f);
-    return __ldg(reinterpret_cast<const float4*>(plane + (size_t)h * W + col));
+    const float* p = plane + (size_t)h * W + col;
+    if constexpr (VEC) {
+        return __ldg(reinterpret_cast<const float4*>(p));
+    } else {
+        float4 v;
+        v.x = col + 0 < W ? __ldg(p + 0) : 0.f;
+        v.y = col + 1 < W ? __ldg(p + 1) : 0.f;
+        v.z = col + 2 < W ? __ldg(p + 2) : 0.f;
+        v.w = col + 3 < W ? __ldg(p + 3) : 0.f;
+        return v;
+    }
+}
+template <bool VEC>
+__device__ __forceinline__ void strow(float* __restrict__ dst, int col, int W, const float (&acc)[4]) {
+    if constexpr (VEC) {
+        *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (col + j < W) dst[j] = acc[j];
+    }
 }
 
 // ---- stride 1 -------------------------------------------------------------------------------------
@@ -32,6 +56,7 @@ __device__ __forceinline__ void row_taps1(const float4 v, bool has_l, bool has_r
     acc[3] = fmaf(v.z, w[0], acc[3]); acc[3] = fmaf(v.w, w[1], acc[3]); acc[3] = fmaf(r, w[2], acc[3]);
 }
 
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
@@ -60,12 +85,12 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
     // rows p-1 .. p+U of the current block; `live` only gates memory traffic, every lane runs the shuffles
     float4 cur[U + 2], nxt[U];
 #pragma unroll
-    for (int j = 0; j < U + 2; ++j) cur[j] = live ? ldrow(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < U + 2; ++j) cur[j] = live ? ldrow<VEC>(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
     for (int p = p0; p < p0 + c.RH; p += U) {        // warp-uniform trip count
 #pragma unroll
         for (int j = 0; j < U; ++j) {                  // next block's new rows, in flight during this block's math
             const int h = p + U + 1 + j;
-            nxt[j] = (live && h <= p1) ? ldrow(xp, h, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+            nxt[j] = (live && h <= p1) ? ldrow<VEC>(xp, h, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int j = 0; j < U; ++j) {
@@ -73,8 +98,7 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
             row_taps1(cur[j], has_l, has_r, w[0], acc);
             row_taps1(cur[j + 1], has_l, has_r, w[1], acc);
             row_taps1(cur[j + 2], has_l, has_r, w[2], acc);
-            if (live && p + j < p1 && tag_seen == tag)
-                *reinterpret_cast<float4*>(yp + (size_t)(p + j) * s.W + col) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            if (live && p + j < p1 && tag_seen == tag) strow<VEC>(yp + (size_t)(p + j) * s.W + col, col, s.W, acc);
         }
         cur[0] = cur[U];
         cur[1] = cur[U + 1];
@@ -95,6 +119,7 @@ __device__ __forceinline__ void row_taps2(const float4 a, const float4 b, bool h
     acc[3] = fmaf(b.y, w[0], acc[3]); acc[3] = fmaf(b.z, w[1], acc[3]); acc[3] = fmaf(b.w, w[2], acc[3]);
 }
 
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
@@ -115,27 +140,27 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
     const int p0 = (int)chunk * c.RH;
     const int p1 = min(p0 + c.RH, s.H_out);
     const bool has_l = xq > 0;
-    const bool second_ok = col + 4 < s.W;        // W % 8 == 4: the last strip has only one vector
+    const bool second_ok = col + 4 < s.W;        // the last strip of a row may have only one group of four columns
     float w[3][3];
 #pragma unroll
     for (int i = 0; i < 9; ++i) w[i / 3][i % 3] = live ? __ldg(wpk + (size_t)ch * 9 + i) : 0.f;
     const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
     // input rows 2p-1, 2p, 2p+1 feed output row p; row 2p+1 is row 2(p+1)-1 of the next output
-    float4 ta = live ? ldrow(xp, 2 * p0 - 1, s.H, s.W, col) : z4;
-    float4 tb = (live && second_ok) ? ldrow(xp, 2 * p0 - 1, s.H, s.W, col + 4) : z4;
+    float4 ta = live ? ldrow<VEC>(xp, 2 * p0 - 1, s.H, s.W, col) : z4;
+    float4 tb = (live && second_ok) ? ldrow<VEC>(xp, 2 * p0 - 1, s.H, s.W, col + 4) : z4;
     float4 ca[2], cb[2], na[2], nb[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-        ca[j] = live ? ldrow(xp, 2 * p0 + j, s.H, s.W, col) : z4;
-        cb[j] = (live && second_ok) ? ldrow(xp, 2 * p0 + j, s.H, s.W, col + 4) : z4;
+        ca[j] = live ? ldrow<VEC>(xp, 2 * p0 + j, s.H, s.W, col) : z4;
+        cb[j] = (live && second_ok) ? ldrow<VEC>(xp, 2 * p0 + j, s.H, s.W, col + 4) : z4;
     }
     for (int p = p0; p < p0 + c.RH; ++p) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {                  // rows of the next output, in flight during this one's math
             const int h = 2 * (p + 1) + j;
             const bool need = live && (p + 1 < p1);
-            na[j] = need ? ldrow(xp, h, s.H, s.W, col) : z4;
-            nb[j] = (need && second_ok) ? ldrow(xp, h, s.H, s.W, col + 4) : z4;
+            na[j] = need ? ldrow<VEC>(xp, h, s.H, s.W, col) : z4;
+            nb[j] = (need && second_ok) ? ldrow<VEC>(xp, h, s.H, s.W, col + 4) : z4;
         }
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         row_taps2(ta, tb, has_l, w[0], acc);
@@ -164,15 +189,14 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
 bool dw_supported(const Shape& s) {
     if (!(s.KH == 3 && s.KW == 3 && s.dilation == 1 && s.pad == 1 && (s.stride == 1 || s.stride == 2))) return false;
     if (!(s.Cg == 1 && s.Kg == 1)) return false;
-    if (s.W % 4 != 0) return false;
-    const int xq = s.stride == 1 ? s.W / 4 : (s.W + 7) / 8;
+    const int xq = s.stride == 1 ? (s.W + 3) / 4 : (s.W + 7) / 8;
     if (xq > 32) return false;
     return (unsigned long long)s.N * s.C_in * s.H_out < (1ull << 30);
 }
 
 DwCfg dw_config(const Shape& s, int sm_count) {
     DwCfg c;
-    c.XQ = s.stride == 1 ? s.W / 4 : (s.W + 7) / 8;
+    c.XQ = s.stride == 1 ? (s.W + 3) / 4 : (s.W + 7) / 8;
     c.subs = 32 / c.XQ;
     // rows per thread: long strips amortise the two halo rows, short ones give more parallelism; aim for
     // at least ~6 waves of 1024 threads per SM
@@ -193,10 +217,15 @@ cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float
                        cudaStream_t st) {
     const DwCfg c = dw_config(s, sm_count);
     const uint32_t tag = pack_tag(s, GCONV_VARIANT_DIRECT_TILED);
-    if (s.stride == 1)
-        dw_stream_s1_kernel<<<c.blocks, 256, 0, st>>>(s, c, x, reinterpret_cast<const uint32_t*>(packed), y, status, tag);
-    else
-        dw_stream_s2_kernel<<<c.blocks, 256, 0, st>>>(s, c, x, reinterpret_cast<const uint32_t*>(packed), y, status, tag);
+    const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed);
+    const bool vec = (s.W % 4 == 0);
+    if (s.stride == 1) {
+        if (vec) dw_stream_s1_kernel<true><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        else dw_stream_s1_kernel<false><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+    } else {
+        if (vec) dw_stream_s2_kernel<true><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        else dw_stream_s2_kernel<false><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+    }
     return cudaGetLastError();
 }
 

@@ -134,3 +134,11 @@ SWEEP_GROUPS = (1, 2, 4, 8, 16, 32, 64, 128, 256)
 def sweep_layers(N: int = 32) -> List[Layer]:
     """Group-count sweep to depthwise: 256->256 @56x56, 3x3, stride 1, pad 1."""
     return [Layer("sweep_256@56_g%d" % g, N, 256, 56, 56, 256, groups=g) for g in SWEEP_GROUPS]
+
+
+def mobilenetv2_dw_layers(N: int = 64) -> List[Layer]:
+    """MobileNetV2-shaped depthwise 3x3 layers at 224x224 input (the paper's third network, whose default
+    architecture is the G(N) model): expansion widths 32...960 at spatial 112...7, stride 1 and 2."""
+    mk = lambda C, HW, s: Layer("mbv2_dw_%d@%d%s" % (C, HW, "s2" if s == 2 else ""), N, C, HW, HW, C, stride=s, groups=C)
+    return [mk(32, 112, 1), mk(96, 112, 2), mk(144, 56, 1), mk(144, 56, 2), mk(192, 28, 1), mk(192, 28, 2),
+            mk(384, 14, 1), mk(576, 14, 1), mk(576, 14, 2), mk(960, 7, 1)]

@@ -8,7 +8,8 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
-from paper_2006_09791_b200.workloads import Layer, config0, resnet34_layers, resnext_layers, sweep_layers, wrn_stack
+from paper_2006_09791_b200.workloads import (Layer, config0, mobilenetv2_dw_layers, resnet34_layers, resnext_layers,
+                                             sweep_layers, wrn_stack)
 
 from golden_io import load_case
 from gpu_util import check_layer, rel_err, run_layer
@@ -68,6 +69,8 @@ ODD_SHAPES = [
     (2, 6, 30, 28, 6, 3, 3, 2, 1, 1, 6), (1, 40, 5, 4, 40, 3, 3, 1, 1, 1, 40), (2, 7, 3, 8, 7, 3, 3, 2, 1, 1, 7),
     (3, 16, 14, 14, 32, 3, 3, 2, 1, 1, 2), (2, 8, 7, 7, 8, 3, 3, 1, 1, 1, 1), (1, 32, 9, 30, 32, 3, 3, 1, 1, 1, 4),
     (2, 24, 5, 6, 24, 3, 3, 1, 1, 1, 3), (1, 16, 21, 50, 16, 3, 3, 2, 1, 1, 2), (2, 8, 3, 126, 8, 3, 3, 1, 1, 1, 1),
+    (2, 9, 14, 14, 9, 3, 3, 1, 1, 1, 9), (1, 5, 7, 7, 5, 3, 3, 1, 1, 1, 5), (2, 6, 15, 13, 6, 3, 3, 2, 1, 1, 6),
+    (1, 4, 9, 250, 4, 3, 3, 2, 1, 1, 4), (1, 3, 6, 127, 3, 3, 3, 1, 1, 1, 3),
     (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
 ]
 
@@ -105,6 +108,12 @@ def test_resnext_shapes():
 def test_sweep_to_depthwise_small_batch():
     for L in sweep_layers(N=1):
         check_layer(L)
+
+
+def test_mobilenetv2_depthwise_shapes():
+    for L in mobilenetv2_dw_layers(N=2):
+        check_layer(L)
+        check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC)
 
 
 def test_pack_mismatch_is_reported_not_fatal():
