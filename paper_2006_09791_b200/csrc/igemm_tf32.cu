@@ -161,6 +161,20 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 
+// tile index -> (gn = group * NT + filter tile, mt = pixel tile).  With resident weights the pixel tile runs
+// fastest (a CTA keeps its weights across consecutive tiles); with streamed weights the filter tile runs fastest, so
+// the NT tiles that read the same input block run at the same time and the re-reads hit L2 instead of HBM.
+__device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, uint32_t& gn, uint32_t& mt) {
+    if (c.nt_fast) {
+        uint32_t gm, nt, g;
+        c.div_nt.divmod(tile, gm, nt);
+        c.div_mt.divmod(gm, g, mt);
+        gn = g * (uint32_t)c.NT + nt;
+    } else {
+        c.div_mt.divmod(tile, gn, mt);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xmap4, const Shape s,
                   const IgemmCfg c,
@@ -241,7 +255,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         }
         for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
             uint32_t gn, mt;
-            c.div_mt.divmod((uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
+            tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
             uint32_t gq, ntq;
             c.div_nt.divmod(gn, gq, ntq);
             const int g = (int)gq;
@@ -364,7 +378,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             for (int tile = blockIdx.x; tile < c.num_tiles && ok;
                  tile += gridDim.x, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
                 uint32_t gn, mt;
-                c.div_mt.divmod((uint32_t)tile, gn, mt);
+                tile_coords(c, (uint32_t)tile, gn, mt);
                 const bool mine = (tcount & 1) == mslot;
                 if (c.b_res && (int)gn != cur_gn) {
                     // the previous weight buffer is free once every MMA this warp issued so far has completed
@@ -433,7 +447,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
              tile += gridDim.x, tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
             if (tpar != egroup) continue;              // the other group's tile
             uint32_t gn, mt;
-            c.div_mt.divmod((uint32_t)tile, gn, mt);
+            tile_coords(c, (uint32_t)tile, gn, mt);
             uint32_t n, i;
             int f;
             bool valid;
@@ -731,6 +745,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
     const uint32_t b_tile = 3u * c.chunks * blk;
     c.b_res = b_tile <= 40u * 1024u ? 1 : 0;          // keep a (group, filter tile)'s weights resident, double buffered
+    c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
     c.bres_stride = (b_tile + 1023u) & ~1023u;
     const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
     c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
