@@ -161,6 +161,24 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# multi-rank helpers (replicas only: ranks share nothing but the clock)
+def reduce_max_over_ranks(value, world, device=None):
+    """Largest `value` over all ranks (the job is as slow as its slowest replica)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(flops_per_rank_step, world, ms_max):
+    """Whole-job throughput in GFLOP/s: every replica does the same step, the clock is the slowest rank's."""
+    return world * flops_per_rank_step / (ms_max * 1e-3) / 1e9
+
+
+# ------------------------------------------------------------------------------------------------
 # GPU arm
 class Instance:
     """One layer instance of the step: descriptor, packed weights, its own x and y buffers."""
@@ -211,6 +229,54 @@ def time_layer(torch, gconv, L, stream, reps=40, min_cycle_bytes=2 * L2_BYTES + 
         return statistics.median(times), gconv.gconv_variant(d)
     finally:
         gconv.gconv_desc_destroy(d)
+
+
+def chained_stack_ms(torch, gconv, groups, stream, reps=50):
+    """Batch-1 inference over the 18-layer stack as a real chain (each layer reads the previous layer's output),
+    replayed as one CUDA graph: ms per pass.  This is the shape of the paper's whole-network timings (N = 1),
+    restricted to the grouped 3x3 layers."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    layers = []
+    for L in wl.wrn_stack(groups, 1):
+        layers.extend([L] * L.repeat)
+    descs, wps, bufs = [], [], []
+    x0, _ = synth.make_layer_tensors(1, layers[0].C_in, layers[0].H, layers[0].W, layers[0].C_out, 3, 3, groups, 3)
+    bufs.append(torch.from_numpy(x0).to(dev).reshape(-1))
+    try:
+        for i, L in enumerate(layers):
+            d = gconv.gconv_desc_create(*L.desc_args())
+            descs.append(d)
+            _, w = synth.make_layer_tensors(1, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, 100 + i)
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp, stream)
+            wps.append(wp)
+            bufs.append(torch.empty(L.y_elems, dtype=torch.float32, device=dev))
+
+        def run():
+            for i, d in enumerate(descs):
+                gconv.gconv_forward(d, bufs[i], wps[i], bufs[i + 1], stream)
+
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                run()
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                run()
+            graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            stream.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+        for d in descs:
+            assert gconv.gconv_last_status(d, stream) == 0
+        return e0.elapsed_time(e1) / reps
+    finally:
+        for d in descs:
+            gconv.gconv_desc_destroy(d)
 
 
 def layer_row(L, ms, variant, peaks, gconv):
@@ -296,11 +362,7 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max_over_ranks(ms, world, dev)
 
     # ---- device-resident timing: the step as one CUDA graph ----------------------------------------
     with torch.cuda.stream(stream):
@@ -396,6 +458,7 @@ def run_ours(args):
                 ms, v = time_layer(torch, gconv, L, stream, reps=20)
                 sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
             extra["sweep_layers"] = sweep_rows
+            extra["stack_n1_chained_ms_by_groups"] = {str(g): chained_stack_ms(torch, gconv, g, stream) for g in wl.WRN_GROUPS}
 
     # ---- CPU baseline (rank 0, N=1 only) -----------------------------------------------------------
     cpu = None
@@ -407,7 +470,7 @@ def run_ours(args):
                "sample": "the 18-layer stack at N=%d (of %d) for every group count, oracle as it stands" % (CPU_LEG_BATCH, BATCH)}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": world * step_flops / (ms_dev * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+        line = {"metric": METRIC, "value": aggregate_value(step_flops, world, ms_dev), "unit": UNIT, "n_gpus": world,
                 "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_dev, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32+tf32", "data": "synthetic",
                 "config": {"workload": WORKLOAD, "layers_per_step": len(insts), "batch": BATCH, "groups": list(wl.WRN_GROUPS),
@@ -415,7 +478,7 @@ def run_ours(args):
                            "l2": "every layer instance owns its x/y buffers: %.2f GB cycled per step > 126 MB L2"
                                  % ((h2d + d2h) / 1e9)},
                 "clocks": clocks,
-                "e2e": {"value": world * step_flops / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+                "e2e": {"value": aggregate_value(step_flops, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
                 "gpu_launches": launches_per_step * args.steps,
                 "cpu_baseline": cpu, "layers": rows}
