@@ -39,9 +39,10 @@ BATCH = 128
 CPU_SAMPLE_BATCH = 8      # batch of the reference arm's per-step sample
 CPU_LEG_BATCH = 32        # batch of the cpu_baseline leg of the GPU arm
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes one launch of the dominant kernel moves on average over the step, from the ncu capture summarised in
-# profiles/bench_wrn_stack_launch_list.md (reads only: ncu attributes the write-back of y to no kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.67e6}
+# DRAM bytes one launch of the dominant kernel moves on average over the step, from an ncu launch-list capture of
+# `bench.py --steps 2 --warmup 3 --no-cpu --no-layers` with the dram__bytes_read/write metrics (summary kept under
+# profiles/; reads only: ncu attributes the later write-back of y to no kernel).
+NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.68e6}
 
 
 def load_peaks():

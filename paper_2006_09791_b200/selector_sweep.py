@@ -1,7 +1,7 @@
 """Times every supported kernel variant on a grid of layers; the table it prints is what the
 selector's rule in csrc/gconv_api.cu (select_variant) is derived from.
 
-    python -m paper_2006_09791_b200.selector_sweep [--quick] > table.md
+    python -m paper_2006_09791_b200.selector_sweep [--quick] > table.txt
 
 Each cell is the median per-launch time (µs, cold L2: launches rotate over buffers that cycle more
 than twice the L2) of gconv_forward with that variant forced; `auto` names the selector's choice.
