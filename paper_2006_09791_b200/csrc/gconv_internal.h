@@ -111,7 +111,7 @@ struct IgemmCfg {
     int merge, groups, Cg, Kg;   // adjacent groups presented as one (block-diagonal filters); sizes after merging
     int CK, chunks;          // channels per pipeline stage, stages per vertical tap
     int nr, nseg, wseg;      // vertical taps served by one stage (1 or 3), segments per stage, segments per image row
-    int b_res;               // weights of a (group, filter tile) stay resident in shared memory
+    int b_res;               // resident weight buffers in shared memory: 0 (weights stream with the stages), 1 or 2
     int nt_fast;             // tile order: filter tile fastest (streamed weights) instead of pixel tile fastest
     uint32_t bres_stride;    // bytes between the two resident weight buffers
     int Kt, NT, Np;          // filters per tile, filter tiles per group, MMA N (3*Kt padded to 16)

@@ -46,6 +46,7 @@ constexpr int kThreads = 32 * (kEpi2First + kEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr int kMaxDynSmem = 214 * 1024;   // 227 KB per CTA minus the static control block and exchange buffers
 
 struct __align__(8) SharedCtl {
     unsigned long long full[8];
@@ -235,7 +236,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     const uint32_t blk_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;   // weights of one (chunk, tap)
     const uint32_t b_tile_bytes = 3u * (uint32_t)c.chunks * blk_bytes;   // weights of one (group, filter tile)
     const uint32_t bres_base = smem_base;                                // two resident weight buffers (if b_res)
-    const uint32_t stage_base = smem_base + (c.b_res ? 2u * c.bres_stride : 0u);
+    const uint32_t stage_base = smem_base + (uint32_t)c.b_res * c.bres_stride;   // b_res = number of resident weight buffers
     const int HW = s.H * s.W;
     const size_t OHW = (size_t)s.H_out * s.W_out;
 
@@ -261,7 +262,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
             if (c.b_res && (int)gn != cur_gn) {
-                const uint32_t bb = switches & 1, use = switches >> 1;
+                const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
                 if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
                 const uint32_t bar = smem_u32(&ctl.b_full[bb]);
                 if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
@@ -346,11 +347,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
                     if (mbar_try_wait(bar, (j / c.stages) & 1)) break;
             }
-            for (uint32_t i = 0; i < 2 && i < switches; ++i) {
+            for (uint32_t i = 0; i < (uint32_t)c.b_res && i < switches; ++i) {
                 const uint32_t j = switches - 1 - i;
-                const uint32_t bar = smem_u32(&ctl.b_full[j & 1]);
+                const uint32_t bar = smem_u32(&ctl.b_full[c.b_res == 2 ? (j & 1) : 0u]);
+                const uint32_t par = (c.b_res == 2 ? (j >> 1) : j) & 1;
                 for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
-                    if (mbar_try_wait(bar, (j >> 1) & 1)) break;
+                    if (mbar_try_wait(bar, par)) break;
             }
         }
     } else if (warp == 1 || warp == kMmaWarp2) {
@@ -383,11 +385,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 if (c.b_res && (int)gn != cur_gn) {
                     // the previous weight buffer is free once every MMA this warp issued so far has completed
                     // (the barrier counts both issuing warps)
-                    if (switches > 0) umma_commit(smem_u32(&ctl.b_free[(switches - 1) & 1]));
+                    const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
+                    if (switches > 0) umma_commit(smem_u32(&ctl.b_free[c.b_res == 2 ? ((switches - 1) & 1) : 0u]));
                     // Both warps observe every fill of a weight buffer, in order, even when the tiles that
                     // use it are the other warp's: a parity wait is only meaningful one phase at a time.
-                    if (!mbar_wait(smem_u32(&ctl.b_full[switches & 1]), (switches >> 1) & 1, abort_flag, status, 700)) break;
-                    bres_addr = bres_base + (switches & 1) * c.bres_stride;
+                    if (!mbar_wait(smem_u32(&ctl.b_full[bb]), use & 1, abort_flag, status, 700)) break;
+                    bres_addr = bres_base + bb * c.bres_stride;
                     cur_gn = (int)gn;
                     ++switches;
                 }
@@ -744,17 +747,26 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     c.div_nt = make_fastdiv((uint32_t)c.NT);
     const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
     const uint32_t b_tile = 3u * c.chunks * blk;
-    c.b_res = b_tile <= 40u * 1024u ? 1 : 0;          // keep a (group, filter tile)'s weights resident, double buffered
+    // Weights of a (group, filter tile) stay resident in shared memory when they fit: two buffers (the next group's
+    // weights load while the current group computes) up to 40 KB each, one buffer (the switch waits for the MMAs
+    // of the outgoing group) up to 144 KB; larger filter banks stream with the input stages.
+    c.b_res = b_tile <= 40u * 1024u ? 2 : (b_tile <= 144u * 1024u ? 1 : 0);
+    {   // a single resident buffer must still leave room for two input stages
+        const uint32_t a_only = ((uint32_t)c.nseg * c.CK * 128u + 1023u) & ~1023u;
+        if (c.b_res == 1 && ((b_tile + 1023u) & ~1023u) + 2u * a_only + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
+        // loading a large filter bank up front only pays when a CTA reuses it over several pixel tiles
+        if (c.b_res == 1 && c.MT < 4 * sm_count) c.b_res = 0;
+    }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
     c.bres_stride = (b_tile + 1023u) & ~1023u;
     const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
     c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
-    const uint32_t budget = 196u * 1024u - (c.b_res ? 2u * c.bres_stride : 0u);
+    const uint32_t budget = 200u * 1024u - (uint32_t)c.b_res * c.bres_stride;
     int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
     if (st < 2) st = 2;
     c.stages = st;
-    c.smem_bytes = (size_t)c.stages * c.stage_bytes + (c.b_res ? 2u * c.bres_stride : 0u) + 1024;
+    c.smem_bytes = (size_t)c.stages * c.stage_bytes + (size_t)c.b_res * c.bres_stride + 1024;
     c.grid = c.num_tiles < sm_count ? c.num_tiles : sm_count;
     return c;
 }
@@ -835,7 +847,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(igemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(igemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
