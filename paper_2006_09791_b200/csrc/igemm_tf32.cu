@@ -257,83 +257,76 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
-            uint32_t gq, ntq;
-            c.div_nt.divmod(gn, gq, ntq);
+            uint32_t gq = gn, ntq = 0;
+            if (c.NT > 1) c.div_nt.divmod(gn, gq, ntq);
             const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
-            if (c.b_res && (int)gn != cur_gn) {
-                const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
-                if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
-                const uint32_t bar = smem_u32(&ctl.b_full[bb]);
-                if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
-                __syncwarp();
-                for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
-                    bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
-                cur_gn = (int)gn;
-                ++switches;
-            }
-            // this lane's segment: image index and first flat pixel (tap r adds (r-1)*W)
-            int my_n, my_f;
-            if (c.nr == 3) {                               // tile plus halo: contiguous segments of one image
-                uint32_t n, i;
-                if (c.seg_mode) c.div_spi.divmod(mt * 4u, n, i); else c.div_spi.divmod(mt, n, i);
-                my_n = (int)n;
-                my_f = (c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W) + (lane - c.wseg) * 32;
-            } else if (c.seg_mode) {
-                uint32_t n, i;
-                c.div_spi.divmod(mt * 4u + (uint32_t)(lane & 3), n, i);
-                my_n = (int)n < s.N ? (int)n : s.N;        // past the last image: fully out of bounds, zero fill
-                my_f = (int)i * c.seg_fstep;
-            } else {
-                uint32_t n, i;
-                c.div_spi.divmod(mt, n, i);
-                my_n = (int)n;
-                my_f = (int)i * c.R * s.W + 32 * (lane & 3);
-            }
-            const bool issuer = lane < c.nseg;
-            // One 4-D box (32 pixels x CK channels x nseg segments) replaces the per-segment copies whenever the
-            // tile's segments are one contiguous run that stays inside the image plane for the tap at hand; the
-            // plane's first and last tiles (whose halo is out of range and must be zero-filled) keep the
-            // per-segment copies, where out-of-range means out of the plane.
+            const bool switch_b = c.b_res && (int)gn != cur_gn;
+            // Whole-tile copies: a row-box tile is always one 5-D box; a flat tile whose segments are one contiguous run
+            // is one 4-D box for every tap whose run stays inside the image plane.  Everything else (tiles that straddle
+            // images, and the plane's first/last tiles, whose out-of-plane part must be zero-filled) is copied segment
+            // by segment, lane j issuing segment j with its own (image, first pixel).
+            const bool whole = c.rowbox || c.fast4;
             int tile_n = 0, tile_f0 = 0, rb_p0 = 0;
-            bool contiguous = false;
-            if (c.rowbox) {
+            if (whole) {
                 uint32_t n, i;
-                c.div_spi.divmod(mt, n, i);
+                c.div_spi.divmod(c.seg_mode ? mt * 4u : mt, n, i);
                 tile_n = (int)n;
-                rb_p0 = (int)i * c.R;                     // first output row of the tile
-            } else if (c.fast4) {
-                uint32_t n, i;
-                if (c.seg_mode) {
-                    c.div_spi.divmod(mt * 4u, n, i);
-                    tile_f0 = (int)i * 32;
-                } else {
-                    c.div_spi.divmod(mt, n, i);
-                    tile_f0 = (int)i * c.R * s.W;
-                }
-                tile_n = (int)n;
-                contiguous = true;
+                if (c.rowbox) rb_p0 = (int)i * c.R;                              // first output row of the tile
+                else tile_f0 = c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W;    // first flat pixel of the tile
             }
+            int my_n = 0, my_f = 0;
+            bool have_lane_coords = false;
             int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
                 if (!mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
+                const int chan = g * c.Cg + ch * c.CK;
+                const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
+                const bool box = c.rowbox || (c.fast4 && lo >= 0 && lo + c.nseg * 32 <= HW);
                 if (lane == 0) {
                     mbar_arrive_expect_tx(full, a_bytes + nb);
+                    if (box) {
+                        if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, 0, rb_p0 - 1, tile_n, full);   // rows above/below and columns past W: zero fill
+                        else tma_load_4d(a_dst, &xmap4, lo, chan, 0, tile_n, full);
+                    }
                     if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
                 }
-                __syncwarp();
-                const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
-                if (c.rowbox) {
-                    // one 5-D box: 32 pixels x CK channels x SR row segments x (RT + 2) rows; rows outside the image and
-                    // columns past W are zero-filled by TMA, which is exactly the padding
-                    if (lane == 0) tma_load_5d(a_dst, &xmap4, 0, g * c.Cg + ch * c.CK, 0, rb_p0 - 1, tile_n, full);
-                } else if (contiguous && lo >= 0 && lo + c.nseg * 32 <= HW) {
-                    if (lane == 0) tma_load_4d(a_dst, &xmap4, lo, g * c.Cg + ch * c.CK, 0, tile_n, full);
-                } else if (issuer) {
-                    tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, g * c.Cg + ch * c.CK, my_n, full);
+                if (!box) {
+                    if (!have_lane_coords) {
+                        uint32_t n, i;
+                        if (c.nr == 3) {                   // tile plus halo: contiguous segments of one image
+                            c.div_spi.divmod(c.seg_mode ? mt * 4u : mt, n, i);
+                            my_n = (int)n;
+                            my_f = (c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W) + (lane - c.wseg) * 32;
+                        } else if (c.seg_mode) {
+                            c.div_spi.divmod(mt * 4u + (uint32_t)(lane & 3), n, i);
+                            my_n = (int)n < s.N ? (int)n : s.N;   // past the last image: fully out of bounds, zero fill
+                            my_f = (int)i * c.seg_fstep;
+                        } else {
+                            c.div_spi.divmod(mt, n, i);
+                            my_n = (int)n;
+                            my_f = (int)i * c.R * s.W + 32 * (lane & 3);
+                        }
+                        have_lane_coords = true;
+                    }
+                    __syncwarp();                          // the barrier is armed before any lane's copy can complete on it
+                    if (lane < c.nseg) tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, chan, my_n, full);
+                }
+                if (ks == 0 && switch_b) {
+                    // New (group, filter tile): its weights go to the free resident buffer.  Issued after the tile's
+                    // first input copy, which has the longer way to come (HBM); the weights are usually in L2.
+                    const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
+                    if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&ctl.b_full[bb]);
+                    if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
+                    __syncwarp();
+                    for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                        bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
+                    cur_gn = (int)gn;
+                    ++switches;
                 }
                 if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
