@@ -82,3 +82,35 @@ def test_group_sweep_at_batch_32(idx):
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(78, idx), L.x_dist)
     y, v = _run_full(L, x, w, use_graph=True)
     _check_samples(L, y, x, w, v, _samples(L, 3 if L.groups == 1 else 6, idx))
+
+
+def test_more_than_2_to_31_elements():
+    """Maximum sizes: x and y each hold more than 2^31 elements, so every 32-bit index in the path would wrap.
+    The batch is a two-image block repeated on the device; slices are checked against the oracle on that block."""
+    from paper_2006_09791_b200.workloads import Layer
+    for groups, C in ((2, 128), (128, 128)):          # tensor-core variant and depthwise stream kernel
+        N = 4100 if groups == 2 else 4400
+        L = Layer("huge_g%d" % groups, N, C, 64, 64, C, groups=groups)
+        assert L.x_elems > 2 ** 31 and L.y_elems > 2 ** 31
+        dev = torch.device("cuda:0")
+        xb, w = synth.make_layer_tensors(2, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, synth.layer_seed(79, groups))
+        d = gconv.gconv_desc_create(*L.desc_args())
+        try:
+            x = torch.from_numpy(xb).to(dev).repeat(N // 2, 1, 1, 1)
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            y = torch.full((L.y_elems,), float("nan"), dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
+            gconv.gconv_forward(d, x, wp, y)
+            assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+            v = gconv.gconv_variant(d)
+            tol = gconv.VARIANT_TOLERANCE[v]
+            yv = y.view(N, L.C_out, L.H_out, L.W_out)
+            assert bool(torch.isfinite(yv[::97]).all()) and bool(torch.isfinite(yv[-3:]).all())
+            for n, g in [(0, 0), (N - 1, groups - 1), (N // 2 + 1, groups // 2), (2049, 1), (N - 2, 0)]:
+                ref = oracle.gconv_ref(xb[n % 2:n % 2 + 1, g * L.Cg:(g + 1) * L.Cg], w[g * L.Kg:(g + 1) * L.Kg], 1, 1, 1, 1, threads=16)[0]
+                got = yv[n, g * L.Kg:(g + 1) * L.Kg].cpu().numpy().astype(np.float64)
+                assert np.max(np.abs(got - ref)) <= tol * max(np.max(np.abs(ref)), 1e-30), (L.name, n, g)
+            del x, y, yv
+            torch.cuda.empty_cache()
+        finally:
+            gconv.gconv_desc_destroy(d)
