@@ -71,6 +71,8 @@ ODD_SHAPES = [
     (2, 24, 5, 6, 24, 3, 3, 1, 1, 1, 3), (1, 16, 21, 50, 16, 3, 3, 2, 1, 1, 2), (2, 8, 3, 126, 8, 3, 3, 1, 1, 1, 1),
     (2, 9, 14, 14, 9, 3, 3, 1, 1, 1, 9), (1, 5, 7, 7, 5, 3, 3, 1, 1, 1, 5), (2, 6, 15, 13, 6, 3, 3, 2, 1, 1, 6),
     (1, 4, 9, 250, 4, 3, 3, 2, 1, 1, 4), (1, 3, 6, 127, 3, 3, 3, 1, 1, 1, 3),
+    (2, 40, 12, 16, 72, 3, 3, 1, 1, 1, 1), (1, 24, 28, 28, 88, 3, 3, 1, 1, 1, 1), (2, 48, 8, 8, 120, 3, 3, 2, 1, 1, 3),
+    (1, 160, 16, 32, 160, 3, 3, 1, 1, 1, 5), (3, 36, 6, 44, 36, 3, 3, 1, 1, 1, 9), (1, 12, 64, 64, 12, 3, 3, 1, 1, 1, 6),
     (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
 ]
 
