@@ -120,6 +120,7 @@ struct IgemmCfg {
     int seg_fstep;           // flat-pixel step between consecutive segments of an image
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int nacc;                // accumulator buffers in the TMEM ring
+    int issuers;             // MMA-issuing warps (2 or 4), one per accumulator buffer
     int fast4;               // a second tensor map for whole-tile copies is available
     int padded, Hv, Wv;      // the kernel computes on a zero-padded copy of x; valid extent of the plane
     int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)

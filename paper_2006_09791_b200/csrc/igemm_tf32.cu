@@ -26,7 +26,8 @@
 // All groups and all images run in one persistent launch: the tile index enumerates
 // (group, filter tile, pixel tile), one CTA per SM walks it.
 //
-// Warp roles: warp 0 = TMA producer, warps 1 and 10 = single-thread MMA issuers for alternate tiles (warp 1 owns TMEM),
+// Warp roles: warp 0 = TMA producer, warps 1, 10 (and 19, 20 when four accumulators fit) = single-thread MMA issuers
+// taking tiles in turn, each with its own accumulator buffer (warp 1 owns the TMEM allocation),
 // warps 2..9 and 11..18 = two epilogue groups for alternate tiles (TMEM lane quarter = warp_id % 4).
 // Every mbarrier wait is bounded: when a
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
@@ -42,7 +43,8 @@ namespace {
 constexpr int kEpiWarps = 8;             // warps of one epilogue group: two per TMEM lane quarter, each takes half of the filters
 constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the first is warp 1)
 constexpr int kEpi2First = kMmaWarp2 + 1;    // first warp of the second epilogue group
-constexpr int kThreads = 32 * (kEpi2First + kEpiWarps);
+constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issuing warps (used when four accumulators fit)
+constexpr int kThreads = 32 * (kMmaWarp3 + 2);
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 constexpr uint32_t kSpinLimit = 1u << 20;
@@ -208,7 +210,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl.b_full[i]), 1);
-            mbar_init(smem_u32(&ctl.b_free[i]), 2);
+            mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
         }
         ctl.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -348,13 +350,13 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                     if (mbar_try_wait(bar, par)) break;
             }
         }
-    } else if (warp == 1 || warp == kMmaWarp2) {
+    } else if (warp == 1 || warp == kMmaWarp2 || warp >= kMmaWarp3) {
         // ---------------------------------------------------------------- MMA issuers
         // Two warps issue alternate tiles (each owns one TMEM buffer), so the barrier waits and descriptor
         // set-up of one tile hide behind the other warp's MMAs.  Both walk every tile to keep the stage ring
         // and the weight-buffer switches in step.
-        const uint32_t mslot = warp == 1 ? 0u : 1u;
-        if (lane == 0) {
+        const uint32_t mslot = warp == 1 ? 0u : (warp == kMmaWarp2 ? 1u : 2u + (uint32_t)(warp - kMmaWarp3));
+        if (lane == 0 && mslot < (uint32_t)c.issuers) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((uint32_t)(c.Np >> 3) << 17) |
                                    ((128u >> 4) << 24);
             const uint32_t b_lbo = (uint32_t)(c.Np >> 3) * 128u;   // next 4-channel core matrix along K
@@ -367,14 +369,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             int stage = 0;
             uint32_t ph = 0;
             uint32_t buf = 0, bph = 0;      // accumulator ring position of the current tile and its pass parity
+            uint32_t turn = 0;              // which issuing warp's turn the current tile is
             int cur_gn = -1;
             uint32_t bres_addr = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < c.num_tiles && ok;
-                 tile += gridDim.x, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
+                 tile += gridDim.x, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u),
+                     turn = (turn + 1 == (uint32_t)c.issuers ? 0u : turn + 1)) {
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
-                const bool mine = (tcount & 1) == mslot;
+                const bool mine = turn == mslot;
                 if (c.b_res && (int)gn != cur_gn) {
                     // the previous weight buffer is free once every MMA this warp issued so far has completed
                     // (the barrier counts both issuing warps)
@@ -733,6 +737,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     }
     c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
+    c.issuers = c.nacc;                                // MMA-issuing warps: one per accumulator buffer
     c.num_tiles = c.groups * c.NT * c.MT;
     c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)(c.seg_mode ? c.SPI : c.RB));
