@@ -198,22 +198,27 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     const uint32_t smem_base = smem_u32(smem);
     volatile int* abort_flag = &ctl.abort_flag;
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < c.stages; ++i) {
-            mbar_init(smem_u32(&ctl.full[i]), 1);
-            mbar_init(smem_u32(&ctl.empty[i]), 1);
-        }
-        for (int i = 0; i < kMaxAcc; ++i) {
+    // barrier set-up, one barrier per thread of the last warps (warp 1 is busy allocating TMEM meanwhile)
+    {
+        const int t = (int)threadIdx.x - 64;
+        if (t >= 0 && t < 8) {
+            if (t < c.stages) {
+                mbar_init(smem_u32(&ctl.full[t]), 1);
+                mbar_init(smem_u32(&ctl.empty[t]), 1);
+            }
+        } else if (t >= 8 && t < 8 + kMaxAcc) {
+            const int i = t - 8;
             mbar_init(smem_u32(&ctl.tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl.tmem_empty[i]), kEpiWarps);
             mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
-        }
-        for (int i = 0; i < 2; ++i) {
+        } else if (t >= 16 && t < 18) {
+            const int i = t - 16;
             mbar_init(smem_u32(&ctl.b_full[i]), 1);
             mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
+        } else if (t == 18) {
+            ctl.abort_flag = 0;
         }
-        ctl.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (t >= 0 && t < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
