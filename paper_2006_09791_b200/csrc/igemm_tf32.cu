@@ -187,9 +187,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     __shared__ float xchg[kMaxAcc][4][2][64];
 
     // Programmatic dependent launch: let the next kernel in the stream be scheduled as SMs free up, and run this
-    // kernel's own set-up (barriers, TMEM) while the previous kernel drains; nothing below touches global memory
-    // until griddepcontrol.wait has returned, i.e. until the previous kernel's writes are complete and visible.
+    // kernel's own set-up (barriers, TMEM) while the previous kernel drains.  Before griddepcontrol.wait has
+    // returned (the previous kernel's writes complete and visible) the only global memory read is the tag of the
+    // packed weights: they are written by the packing kernel, which never releases its dependents early, so it
+    // had completed before any later kernel of the stream started.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const uint32_t tag_seen = __ldg(packed);
     const uint8_t* __restrict__ wblocks = reinterpret_cast<const uint8_t*>(packed) + kHeaderBytes;
 
     const int warp = threadIdx.x >> 5;
@@ -231,7 +234,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const bool tag_ok = (packed[0] == tag);   // uniform across the CTA
+    const bool tag_ok = (tag_seen == tag);   // uniform across the CTA
     if (!tag_ok && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 
     // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
