@@ -233,9 +233,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     const bool tag_ok = (tag_seen == tag);   // uniform across the CTA
-    if (!tag_ok && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 
     // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
     // segments of one vertical tap (nr = 1, stages run chunk-major, tap-minor), or the tile plus its
@@ -252,6 +250,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
 
     if (!tag_ok) {
         // wrong weights: no role runs, y stays untouched; fall through to the common exit (TMEM is freed there)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
     } else if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
@@ -262,8 +262,22 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         bool ok = true;
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
-            if (c.fast4) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap4) : "memory");
+            if (c.fast4 || c.rowbox) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap4) : "memory");
         }
+        if (c.b_res && (int)blockIdx.x < c.num_tiles) {
+            // The first tile's resident weights do not depend on the previous kernel: fetch them before waiting for it.
+            uint32_t gn, mt;
+            tile_coords(c, blockIdx.x, gn, mt);
+            const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
+            const uint32_t bar = smem_u32(&ctl.b_full[0]);
+            if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
+            __syncwarp();
+            for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                bulk_load_1d(bres_base + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
+            cur_gn = (int)gn;
+            switches = 1;
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
         for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
@@ -442,6 +456,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         // ---------------------------------------------------------------- epilogue warps
         // Two groups of eight warps take alternate tiles, so one tile's TMEM reads, shuffles and stores overlap
         // the next tile's.  With an even number of accumulators a buffer always belongs to the same group.
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // y may still be read (or written) by the previous kernel
         const int wq = warp & 3;                       // TMEM lane quarter this warp may read
         const uint32_t egroup = warp >= kEpi2First ? 1u : 0u;
         const int half = ((warp - (egroup ? kEpi2First : 2)) >> 2);   // which half of the tile's filters this warp stores
