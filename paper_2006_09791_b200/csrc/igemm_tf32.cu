@@ -303,7 +303,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             bool have_lane_coords = false;
             int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
-                if (!mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                // the first pass over the ring finds every stage free
+                if (it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
