@@ -121,6 +121,10 @@ struct IgemmCfg {
     int need_xchg;           // rows may straddle a warp boundary in the epilogue
     int nacc;                // accumulator buffers in the TMEM ring
     int issuers;             // MMA-issuing warps (2 or 4), one per accumulator buffer
+    int egroups, threads;    // epilogue groups of eight warps (1 or 2) and the block size that goes with them
+    int cps;                 // CTAs per (group, filter tile) when the grid is split into one set per pair, else 0
+    int tmem_cols;           // TMEM columns the CTA allocates (power of two >= nacc * Np)
+    uint32_t xchg_off;       // offset of the edge-lane exchange area in dynamic shared memory
     int fast4;               // a second tensor map for whole-tile copies is available
     int padded, Hv, Wv;      // the kernel computes on a zero-padded copy of x; valid extent of the plane
     int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)

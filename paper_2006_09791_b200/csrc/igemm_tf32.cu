@@ -48,7 +48,7 @@ constexpr int kThreads = 32 * (kMmaWarp3 + 2);
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 constexpr uint32_t kSpinLimit = 1u << 20;
-constexpr int kMaxDynSmem = 214 * 1024;   // 227 KB per CTA minus the static control block and exchange buffers
+constexpr int kMaxDynSmem = 226 * 1024;   // 227 KB per CTA minus the static control block (under 1 KB)
 
 struct __align__(8) SharedCtl {
     unsigned long long full[8];
@@ -184,7 +184,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                   const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
-    __shared__ float xchg[kMaxAcc][4][2][64];
+    static_assert(sizeof(SharedCtl) <= 1024, "control block must leave 226 KB of dynamic shared memory");
 
     // Programmatic dependent launch: let the next kernel in the stream be scheduled as SMs free up, and run this
     // kernel's own set-up (barriers, TMEM) while the previous kernel drains.  Before griddepcontrol.wait has
@@ -200,6 +200,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
     volatile int* abort_flag = &ctl.abort_flag;
+    float (*xchg)[4][2][64] = reinterpret_cast<float (*)[4][2][64]>(smem + c.xchg_off);   // edge-lane exchange (flat row tiles only)
 
     // barrier set-up, one barrier per thread of the last warps (warp 1 is busy allocating TMEM meanwhile)
     {
@@ -225,7 +226,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
-                     "r"(kTmemCols)
+                     "r"((uint32_t)c.tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -234,6 +235,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
     const bool tag_ok = (tag_seen == tag);   // uniform across the CTA
+    // Tiles of this CTA: every gridDim.x-th tile, or -- with resident weights and several (group, filter tile) pairs --
+    // the CTAs split into one set per pair, each set striding over that pair's pixel tiles: no CTA ever switches
+    // weights, and the CTAs of a set still read neighbouring pixels at the same time.
+    int tile_first = (int)blockIdx.x, tile_end = c.num_tiles, tile_step = (int)gridDim.x;
+    if (c.cps > 0) {
+        const int set = (int)blockIdx.x / c.cps;
+        tile_first = set * c.MT + ((int)blockIdx.x - set * c.cps);
+        tile_end = (set + 1) * c.MT;
+        tile_step = c.cps;
+    }
 
     // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
     // segments of one vertical tap (nr = 1, stages run chunk-major, tap-minor), or the tile plus its
@@ -264,10 +275,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
             if (c.fast4 || c.rowbox) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap4) : "memory");
         }
-        if (c.b_res && (int)blockIdx.x < c.num_tiles) {
+        if (c.b_res && tile_first < tile_end) {
             // The first tile's resident weights do not depend on the previous kernel: fetch them before waiting for it.
             uint32_t gn, mt;
-            tile_coords(c, blockIdx.x, gn, mt);
+            tile_coords(c, (uint32_t)tile_first, gn, mt);
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
             const uint32_t bar = smem_u32(&ctl.b_full[0]);
             if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
@@ -278,7 +289,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             switches = 1;
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
-        for (int tile = blockIdx.x; tile < c.num_tiles && ok; tile += gridDim.x) {
+        for (int tile = tile_first; tile < tile_end && ok; tile += tile_step) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
             uint32_t gq = gn, ntq = 0;
@@ -396,8 +407,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             int cur_gn = -1;
             uint32_t bres_addr = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < c.num_tiles && ok;
-                 tile += gridDim.x, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u),
+            for (int tile = tile_first; tile < tile_end && ok;
+                 tile += tile_step, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u),
                      turn = (turn + 1 == (uint32_t)c.issuers ? 0u : turn + 1)) {
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
@@ -467,9 +478,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         const int kbeg = half == 0 ? 0 : kh;
         const int kend = half == 0 ? kh : Kt;
         uint32_t buf = 0, bph = 0, tpar = 0;
-        for (int tile = blockIdx.x; tile < c.num_tiles;
-             tile += gridDim.x, tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
-            if (tpar != egroup) continue;              // the other group's tile
+        for (int tile = tile_first; tile < tile_end;
+             tile += tile_step, tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
+            if (c.egroups == 2 && tpar != egroup) continue;   // the other group's tile
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);
             uint32_t n, i;
@@ -562,7 +573,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
     __syncthreads();
     tc_fence_after();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)c.tmem_cols) : "memory");
     }
 }
 
@@ -678,7 +689,7 @@ bool igemm_supported(const Shape& s) {
     if (ge.Wp > 128) return false;
     if ((long long)ge.Hp * ge.Wp < 32) return false;
     if (s.C_in > 65535 * 8) return false;
-    return true;
+    return igemm_config(s, 148).smem_bytes <= (size_t)kMaxDynSmem;   // the smallest pipeline (two stages) must fit
 }
 
 size_t igemm_scratch_bytes(const Shape& s) {
@@ -769,27 +780,66 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     c.div_nt = make_fastdiv((uint32_t)c.NT);
     const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
     const uint32_t b_tile = 3u * c.chunks * blk;
+    const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
+    const uint32_t xchg_bytes = c.need_xchg ? (uint32_t)(kMaxAcc * 4 * 2 * 64 * sizeof(float)) : 0u;
     // Weights of a (group, filter tile) stay resident in shared memory when they fit: two buffers (the next group's
     // weights load while the current group computes) up to 40 KB each, one buffer (the switch waits for the MMAs
     // of the outgoing group) up to 144 KB; larger filter banks stream with the input stages.
+    c.bres_stride = (b_tile + 1023u) & ~1023u;
     c.b_res = b_tile <= 40u * 1024u ? 2 : (b_tile <= 144u * 1024u ? 1 : 0);
+    if (c.b_res == 2 && c.groups * c.NT == 1) c.b_res = 1;   // a single filter bank: nothing to switch to
     {   // a single resident buffer must still leave room for two input stages
-        const uint32_t a_only = ((uint32_t)c.nseg * c.CK * 128u + 1023u) & ~1023u;
-        if (c.b_res == 1 && ((b_tile + 1023u) & ~1023u) + 2u * a_only + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
+        const uint32_t a_only = (a_bytes + 1023u) & ~1023u;
+        if (c.b_res == 1 && c.bres_stride + 2u * a_only + xchg_bytes + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
         // loading a large filter bank up front only pays when a CTA reuses it over several pixel tiles
-        if (c.b_res == 1 && c.MT < 4 * sm_count) c.b_res = 0;
+        if (c.b_res == 1 && b_tile > 40u * 1024u && c.MT < 4 * sm_count) c.b_res = 0;
+    }
+    c.egroups = 2;
+    c.threads = kThreads;
+    c.tmem_cols = kTmemCols;
+    uint32_t budget_total = 200u * 1024u;
+    // Light configuration, two CTAs per SM: one epilogue group, two accumulators in 256 TMEM columns, one resident
+    // weight buffer and half the shared memory.  The two CTAs hide each other's start-up, barrier and drain
+    // latencies, and a CTA of the next kernel in the stream can start while one of this kernel's is still at work.
+    {
+        const uint32_t light_total = 110u * 1024u;
+        const uint32_t st_bytes = (a_bytes + 1023u) & ~1023u;
+        const int kst = (3 / c.nr) * c.chunks;
+        const bool fits = 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
+                          c.bres_stride + (uint32_t)(kst + 1 < 3 ? 3 : kst + 1) * st_bytes + xchg_bytes + 1024u <= light_total;
+        if (fits) {
+            c.b_res = 1;
+            c.nacc = 2;
+            c.issuers = 2;
+            c.egroups = 1;
+            c.threads = 32 * kEpi2First;       // producer, first MMA warp, first epilogue group, second MMA warp
+            c.tmem_cols = 256;
+            budget_total = light_total - 1024u;
+        }
     }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
-    c.bres_stride = (b_tile + 1023u) & ~1023u;
-    const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
     c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
-    const uint32_t budget = 200u * 1024u - (uint32_t)c.b_res * c.bres_stride;
+    const uint32_t budget = budget_total - (uint32_t)c.b_res * c.bres_stride - xchg_bytes;
     int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
     if (st < 2) st = 2;
     c.stages = st;
-    c.smem_bytes = (size_t)c.stages * c.stage_bytes + (size_t)c.b_res * c.bres_stride + 1024;
-    c.grid = c.num_tiles < sm_count ? c.num_tiles : sm_count;
+    c.xchg_off = (uint32_t)c.stages * c.stage_bytes + (uint32_t)c.b_res * c.bres_stride;
+    c.smem_bytes = (size_t)c.xchg_off + xchg_bytes + 1024;
+    c.grid = c.egroups == 1 ? (c.num_tiles < 2 * sm_count ? c.num_tiles : 2 * sm_count)
+                            : (c.num_tiles < sm_count ? c.num_tiles : sm_count);
+    // With a single resident weight buffer a switch of (group, filter tile) stalls the pipeline, so the CTAs split
+    // into one set per pair and no CTA ever switches (two buffers hide the switch; there the plain order keeps all
+    // SMs busy and balanced).
+    c.cps = 0;
+    {
+        const int n_gn = c.groups * c.NT;
+        if (c.b_res == 1 && n_gn > 1 && c.grid >= n_gn) {
+            c.cps = c.grid / n_gn;                   // CTAs per (group, filter tile)
+            if (c.cps > c.MT) c.cps = c.MT;
+            c.grid = c.cps * n_gn;
+        }
+    }
     return c;
 }
 
@@ -875,7 +925,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     }
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)c.grid);
-    lc.blockDim = dim3(kThreads);
+    lc.blockDim = dim3((unsigned)c.threads);
     lc.dynamicSmemBytes = c.smem_bytes;
     lc.stream = st;
     cudaLaunchAttribute attr[1];
