@@ -133,12 +133,17 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+// One MMA: D[128 x N] (+)= A[128 x 8] * B[8 x N], TF32 in, FP32 accumulate in TMEM.  Each shared-memory descriptor is
+// given as its two 32-bit halves: between MMAs only the low words change.
+__device__ __forceinline__ void umma_tf32_split(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                uint32_t idesc, uint32_t acc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -396,9 +401,18 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             const uint32_t b_lbo = (uint32_t)(c.Np >> 3) * 128u;   // next 4-channel core matrix along K
             const uint32_t b_kstep = 2u * b_lbo;                   // 8 channels
             // descriptors differ only in the start-address field of the low word
-            const uint64_t a_hi = make_desc(0, seg_bytes, 512u, 1u);
-            const uint64_t b_hi = make_desc(0, b_lbo, 128u, 0u);
+            const uint64_t a_desc0 = make_desc(0, seg_bytes, 512u, 1u);
+            const uint64_t b_desc0 = make_desc(0, b_lbo, 128u, 0u);
+            const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), a_lo0 = (uint32_t)a_desc0;   // low word: address (16-byte units) | LBO << 16
+            const uint32_t b_hi = (uint32_t)(b_desc0 >> 32), b_lo0 = (uint32_t)b_desc0;
             const int k8n = c.CK / 8;
+            // 16-byte-unit offsets that do not depend on the tile: the A view of a tap inside a halo stage, the weight
+            // block of a tap, one 8-channel step of B.  Shared-memory addresses stay below 2^18, so adding them to a
+            // low word never carries into the LBO field.
+            const uint32_t view16 = (uint32_t)(c.nr == 3 ? c.wseg : 0) * (seg_bytes >> 4);
+            const uint32_t blk16 = blk_bytes >> 4;
+            const uint32_t bk16 = b_kstep >> 4;
+            const uint32_t b_in_stage16 = a_bytes >> 4;
             uint32_t tcount = 0, switches = 0;
             int stage = 0;
             uint32_t ph = 0;
@@ -441,21 +455,17 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 for (int ks = 0; ks < kstages; ++ks) {
                     if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 300 + stage)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = stage_base + (uint32_t)stage * c.stage_bytes;
-                    for (int rr = 0; rr < c.nr; ++rr) {
-                        // tap r: with a halo stage it is the view that starts r rows (wseg segments per row) in
-                        const uint32_t a_view = a_addr + (c.nr == 3 ? (uint32_t)(rr * c.wseg) * seg_bytes : 0u);
-                        const uint32_t blk = c.nr == 3 ? (uint32_t)(ks * 3 + rr) : (uint32_t)ks;   // (chunk, tap) block
-                        const uint32_t b_addr = c.b_res ? bres_addr + blk * blk_bytes
-                                                        : a_addr + a_bytes + (c.nr == 3 ? (uint32_t)rr * blk_bytes : 0u);
-                        uint64_t adesc = a_hi | (uint64_t)((a_view >> 4) & 0x3FFFu);
-                        uint64_t bdesc = b_hi | (uint64_t)((b_addr >> 4) & 0x3FFFu);
+                    const uint32_t a16 = (stage_base + (uint32_t)stage * c.stage_bytes) >> 4;
+                    // weights of this stage: (chunk, tap) blocks of the resident bank, or the blocks staged behind A
+                    const uint32_t b16 = c.b_res ? (bres_addr >> 4) + (uint32_t)(c.nr == 3 ? ks * 3 : ks) * blk16 : a16 + b_in_stage16;
+                    uint32_t alo = a_lo0 + a16, blo = b_lo0 + b16;
+                    // tap r of a halo stage is the view that starts r rows (wseg segments per row) further in
+                    for (int rr = 0; rr < c.nr; ++rr, alo += view16, blo += blk16) {
+                        uint32_t al = alo, bl = blo;
 #pragma unroll 4
-                        for (int k8 = 0; k8 < k8n; ++k8) {
-                            umma_tf32(d_tmem, adesc, bdesc, idesc, acc);
+                        for (int k8 = 0; k8 < k8n; ++k8, al += 64u, bl += bk16) {
+                            umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc, acc);
                             acc = 1;
-                            adesc += 1024u >> 4;
-                            bdesc += b_kstep >> 4;
                         }
                     }
                     umma_commit(smem_u32(&ctl.empty[stage]));

@@ -85,6 +85,20 @@ def test_odd_shapes_every_variant(cfg):
             check_layer(L, v, seed=7)
 
 
+# Larger row-box layers (several tiles per CTA, ragged last row block, odd number of row blocks, width 56 with two
+# segments per row, stride 2): narrow merged groups, a 64-wide group with one big resident filter bank, streamed filter
+# banks with two and four filter tiles.
+LARGE_ROWBOX_SHAPES = [
+    (12, 128, 56, 56, 128, 3, 3, 1, 1, 1, 4), (44, 64, 56, 56, 64, 3, 3, 1, 1, 1, 1), (40, 256, 30, 28, 256, 3, 3, 1, 1, 1, 2),
+    (24, 64, 54, 56, 64, 3, 3, 2, 1, 1, 8), (90, 32, 28, 40, 32, 3, 3, 1, 1, 1, 2), (11, 128, 56, 52, 256, 3, 3, 1, 1, 1, 1),
+]
+
+
+@pytest.mark.parametrize("cfg", LARGE_ROWBOX_SHAPES)
+def test_large_rowbox_shapes(cfg):
+    check_layer(Layer("rowbox", *cfg), seed=11)
+
+
 @pytest.mark.parametrize("groups", [1, 2, 4, 8, 16])
 def test_wrn_stack_small_batch(groups):
     """Every distinct layer of the WRN-40-2-shaped stack at N = 1 and a ragged N = 3, all variants."""
