@@ -127,6 +127,7 @@ struct IgemmCfg {
     uint32_t xchg_off;       // offset of the edge-lane exchange area in dynamic shared memory
     int fast4;               // a second tensor map for whole-tile copies is available
     int padded, Hv, Wv;      // the kernel computes on a zero-padded copy of x; valid extent of the plane
+    int s2h, lbo_segs;       // stride-2 row tiles (four output rows of one segment, nine staged input rows); segments between M blocks
     int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)
     int num_tiles, stages, grid;
     FastDiv div_nt;                   // (group, filter tile) index -> group

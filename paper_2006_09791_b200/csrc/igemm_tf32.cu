@@ -307,12 +307,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             // images, and the plane's first/last tiles, whose out-of-plane part must be zero-filled) is copied segment
             // by segment, lane j issuing segment j with its own (image, first pixel).
             const bool whole = c.rowbox || c.fast4;
-            int tile_n = 0, tile_f0 = 0, rb_p0 = 0;
+            int tile_n = 0, tile_f0 = 0, rb_row0 = 0, rb_seg = 0;
             if (whole) {
                 uint32_t n, i;
                 c.div_spi.divmod(c.seg_mode ? mt * 4u : mt, n, i);
                 tile_n = (int)n;
-                if (c.rowbox) rb_p0 = (int)i * c.R;                              // first output row of the tile
+                if (c.rowbox && c.s2h) {                 // stride 2: four output rows of one row segment, input rows 2p - 1 .. 2p + 7
+                    const int pb = c.SR == 2 ? (int)(i >> 1) : (int)i;
+                    rb_seg = c.SR == 2 ? (int)(i & 1u) : 0;
+                    rb_row0 = 8 * pb - 1;
+                } else if (c.rowbox) rb_row0 = (int)i * c.R - 1;                 // the row above the tile's first row
                 else tile_f0 = c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W;    // first flat pixel of the tile
             }
             int my_n = 0, my_f = 0;
@@ -330,7 +334,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 if (lane == 0) {
                     mbar_arrive_expect_tx(full, a_bytes + nb);
                     if (box) {
-                        if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, 0, rb_p0 - 1, tile_n, full);   // rows above/below and columns past W: zero fill
+                        if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, rb_seg, rb_row0, tile_n, full);   // rows above/below and columns past W: zero fill
                         else tma_load_4d(a_dst, &xmap4, lo, chan, 0, tile_n, full);
                     }
                     if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
@@ -401,7 +405,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
             const uint32_t b_lbo = (uint32_t)(c.Np >> 3) * 128u;   // next 4-channel core matrix along K
             const uint32_t b_kstep = 2u * b_lbo;                   // 8 channels
             // descriptors differ only in the start-address field of the low word
-            const uint64_t a_desc0 = make_desc(0, seg_bytes, 512u, 1u);
+            const uint64_t a_desc0 = make_desc(0, (uint32_t)c.lbo_segs * seg_bytes, 512u, 1u);   // 32-pixel blocks of M: every segment, or every other one
             const uint64_t b_desc0 = make_desc(0, b_lbo, 128u, 0u);
             const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), a_lo0 = (uint32_t)a_desc0;   // low word: address (16-byte units) | LBO << 16
             const uint32_t b_hi = (uint32_t)(b_desc0 >> 32), b_lo0 = (uint32_t)b_desc0;
@@ -500,9 +504,17 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                 // quarter wq is segment h = wq % SR of row p0 + wq / SR; the last segment of a two-segment row is
                 // shifted left to end at column W, and each column is stored by the segment that holds both of its
                 // horizontal neighbours
+                // (stride 2: quarter wq is output row 4*pb + wq of the tile's one segment, i.e. input row twice that)
                 c.div_spi.divmod(mt, n, i);
-                const int h = c.SR == 2 ? (wq & 1) : 0;
-                const int row = (int)i * c.R + (c.SR == 2 ? (wq >> 1) : wq);
+                int h, row;
+                if (c.s2h) {
+                    const int pb = c.SR == 2 ? (int)(i >> 1) : (int)i;
+                    h = c.SR == 2 ? (int)(i & 1u) : 0;
+                    row = 2 * (4 * pb + wq);
+                } else {
+                    h = c.SR == 2 ? (wq & 1) : 0;
+                    row = (int)i * c.R + (c.SR == 2 ? (wq >> 1) : wq);
+                }
                 const int col = (h ? s.W - 32 : 0) + lane;
                 valid = row < s.H && col < s.W && (c.SR == 1 || (h == 0 ? col <= 30 : col >= 31));
                 f = row * s.W + (col < s.W ? col : s.W - 1);
@@ -766,12 +778,35 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
             c.need_xchg = 0;
         }
     }
+    // Stride 2 on widths 17..62: a tile is four output rows of one 32-column segment.  Its stage holds the nine input
+    // rows 2p-1 .. 2p+7 of that segment; the rows a vertical tap needs are every other one, so tap r is the view that
+    // starts at staged row r with its 32-pixel blocks two rows apart.  Odd input rows are never multiplied or stored
+    // (the odd columns still are: TMA cannot skip elements of the innermost dimension).
+    c.s2h = 0;
+    c.lbo_segs = 1;
+    if (s.stride == 2 && s.W > 16 && s.W <= 62) {
+        c.s2h = 1;
+        c.lbo_segs = 2;
+        c.seg_mode = 0;
+        c.seg_fstep = 32;
+        c.SPI = 0;
+        c.rowbox = 1;
+        c.SR = s.W <= 32 ? 1 : 2;
+        c.R = 4;
+        c.RB = ((s.H_out + 3) / 4) * c.SR;               // tiles per image
+        c.MT = s.N * c.RB;
+        c.need_xchg = 0;
+    }
     // Row halo: when a row is a whole number of 32-pixel segments the three vertical taps are views of
     // one staged block (tile + one row above and below), so the input crosses L2 -> shared memory once.
     c.nr = 1;
     c.nseg = 4;
     c.wseg = 0;
-    if (c.rowbox) {
+    if (c.rowbox && c.s2h) {
+        c.nr = 3;
+        c.wseg = 1;
+        c.nseg = 9;
+    } else if (c.rowbox) {
         c.nr = 3;
         c.wseg = c.SR;
         c.nseg = 4 + 2 * c.SR;
@@ -906,7 +941,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
         const cuuint64_t dims5[5] = {(cuuint64_t)s.W, (cuuint64_t)s.C_in, (cuuint64_t)c.SR, (cuuint64_t)s.H, (cuuint64_t)s.N};
         const cuuint64_t strides5[4] = {HW * 4, c.SR == 2 ? (cuuint64_t)(s.W - 32) * 4 : 128, (cuuint64_t)s.W * 4,
                                         HW * 4 * (cuuint64_t)s.C_in};
-        const cuuint32_t box5[5] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.SR, (cuuint32_t)(c.R + 2), 1};
+        const cuuint32_t box5[5] = {32, (cuuint32_t)c.CK, (cuuint32_t)(c.s2h ? 1 : c.SR), (cuuint32_t)(c.s2h ? 9 : c.R + 2), 1};
         const cuuint32_t estr5[5] = {1, 1, 1, 1, 1};
         if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float*>(x), dims5, strides5, box5, estr5,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
