@@ -851,7 +851,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
         const uint32_t st_bytes = (a_bytes + 1023u) & ~1023u;
         const int kst = (3 / c.nr) * c.chunks;
         const bool fits = 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
-                          c.bres_stride + (uint32_t)(c.s2h ? 2 : (kst + 1 < 3 ? 3 : kst + 1)) * st_bytes + xchg_bytes + 1024u <= light_total;
+                          c.bres_stride + (uint32_t)(kst == 1 ? 2 : kst + 1) * st_bytes + xchg_bytes + 1024u <= light_total;
         if (fits) {
             c.b_res = 1;
             c.nacc = 2;
