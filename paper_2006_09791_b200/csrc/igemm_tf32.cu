@@ -192,15 +192,18 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg;
 };
-constexpr int kFamilies = 6;
+constexpr int kFamilies = 9;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK ch  Kt  Np NT acc iss pad ntf wseg nseg
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32, 1, 32,  96, 1,  2,  2,  0,  0,  0,   4}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32, 1, 32,  96, 1,  2,  2,  0,  0,  1,   6}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32, 1, 32,  96, 1,  2,  2, -1,  0, -1,  -1}     // row boxes, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, 1, 64, 192, 1,  2,  2,  0,  0,  1,   9}     // stride-2 row tiles, 32 -> 64 channels
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32, 1, 32,  96, 1,  2,  2, -1,  0,  1,   9}     // stride-2 row tiles, narrow groups
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,  -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1}     // row boxes, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
@@ -1011,7 +1014,8 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     }
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const Shape, const IgemmCfg, const uint32_t*, float*, Status*, uint32_t);
     static const KernelFn kernels[kFamilies] = {igemm_tf32_kernel<0>, igemm_tf32_kernel<1>, igemm_tf32_kernel<2>,
-                                                igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>};
+                                                igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
+                                                igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
