@@ -42,7 +42,7 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes one launch of the dominant kernel moves on average over the step, from an ncu launch-list capture of
 # `bench.py --steps 2 --warmup 3 --no-cpu --no-layers` with the dram__bytes_read/write metrics (summary kept under
 # profiles/; reads only: ncu attributes the later write-back of y to no kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.68e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.66e6}
 
 
 def load_peaks():
