@@ -190,24 +190,25 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg;
+        nt_fast, wseg, nseg, SR, fast4;
 };
-constexpr int kFamilies = 9;
+constexpr int kFamilies = 10;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1}     // row boxes, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  1}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9,  1,  1}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4,  0, -1}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1}     // row boxes of one segment, narrow groups
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -1015,7 +1016,8 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const Shape, const IgemmCfg, const uint32_t*, float*, Status*, uint32_t);
     static const KernelFn kernels[kFamilies] = {igemm_tf32_kernel<0>, igemm_tf32_kernel<1>, igemm_tf32_kernel<2>,
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
-                                                igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>};
+                                                igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
+                                                igemm_tf32_kernel<9>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
