@@ -132,6 +132,37 @@ def test_mobilenetv2_depthwise_shapes():
         check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC)
 
 
+def _seeded_random_shapes(seed, count):
+    """3x3, pad 1 layers drawn from the sizes the selector, the tilings and the kernel families branch on (plane
+    sizes around the 32-pixel segment and the 128-pixel tile, widths that need padding, narrow and wide groups,
+    unequal Cg and Kg, both strides, ragged batches), each small enough for the oracle."""
+    import random
+    rng = random.Random(seed)
+    out = []
+    while len(out) < count:
+        g = rng.choice([1, 1, 2, 2, 4, 4, 8, 16, 32, 64])
+        cg = rng.choice([1, 2, 4, 8, 8, 16, 16, 32, 32, 64, 128])
+        kg = rng.choice([cg, cg, cg, 2 * cg, max(1, cg // 2), 3 * cg // 2 if cg % 2 == 0 else cg])
+        C, K = g * cg, g * kg
+        if C > 512 or K > 512:
+            continue
+        H = rng.choice([7, 8, 9, 14, 15, 16, 17, 27, 28, 30, 31, 32, 33, 40, 55, 56, 57, 64])
+        W = rng.choice([7, 8, 12, 14, 16, 20, 24, 28, 30, 32, 36, 40, 48, 52, 56, 60, 64, 96, 128])
+        stride = rng.choice([1, 1, 1, 2])
+        macs_per_image = C // g * K * 9 * ((H - 1) // stride + 1) * ((W - 1) // stride + 1)
+        N = min(rng.choice([1, 2, 3, 5, 8, 13, 32, 64, 128, 200]), max(1, int(1.5e9 // macs_per_image)))
+        if N * C * H * W > 40e6:
+            continue
+        out.append((N, C, H, W, K, 3, 3, stride, 1, 1, g))
+    return out
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_seeded_random_shapes(chunk):
+    for i, cfg in enumerate(_seeded_random_shapes(20260 + chunk, 25)):
+        check_layer(Layer("rand%d_%d" % (chunk, i), *cfg), seed=100 * chunk + i)
+
+
 def test_pack_mismatch_is_reported_not_fatal():
     (L,) = config0()
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 5)
