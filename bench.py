@@ -192,7 +192,7 @@ class Instance:
         self.y = torch.empty(L.y_elems, dtype=torch.float32, device=x_dev.device)
 
 
-def time_layer(torch, gconv, L, stream, reps=40, min_cycle_bytes=2 * L2_BYTES + (64 << 20)):
+def time_layer(torch, gconv, L, stream, reps=160, min_cycle_bytes=2 * L2_BYTES + (64 << 20)):
     """Average device time of one gconv_forward launch of layer L with cold L2: launches rotate over
     enough distinct (x, y) buffer pairs that more than twice the L2 is cycled between reuses."""
     dev = torch.device("cuda", torch.cuda.current_device())
