@@ -184,10 +184,105 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
     if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 }
 
+
+// ---- 5x5 depthwise (pad 2) ----------------------------------------------------------------------------
+// The same stream for 5x5 filters: a strip of four output columns reads eight (stride 2: eleven) input columns, its
+// own aligned float4 (stride 2: two) plus two columns from the lane on the left and two (stride 2: one) from the lane
+// on the right; five input rows feed an output row.  Sum order per output: (r, s) as in Algorithm 1.
+__device__ __forceinline__ void row_taps5_s1(const float4 v, bool has_l, bool has_r, const float (&w)[5], float (&acc)[4]) {
+    float l0 = __shfl_up_sync(0xffffffffu, v.z, 1), l1 = __shfl_up_sync(0xffffffffu, v.w, 1);
+    float r0 = __shfl_down_sync(0xffffffffu, v.x, 1), r1 = __shfl_down_sync(0xffffffffu, v.y, 1);
+    if (!has_l) { l0 = 0.f; l1 = 0.f; }
+    if (!has_r) { r0 = 0.f; r1 = 0.f; }
+    const float in[8] = {l0, l1, v.x, v.y, v.z, v.w, r0, r1};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int t = 0; t < 5; ++t) acc[j] = fmaf(in[j + t], w[t], acc[j]);
+}
+__device__ __forceinline__ void row_taps5_s2(const float4 a, const float4 b, bool has_l, bool has_r, const float (&w)[5],
+                                             float (&acc)[4]) {
+    float l0 = __shfl_up_sync(0xffffffffu, b.z, 1), l1 = __shfl_up_sync(0xffffffffu, b.w, 1);
+    float r0 = __shfl_down_sync(0xffffffffu, a.x, 1);
+    if (!has_l) { l0 = 0.f; l1 = 0.f; }
+    if (!has_r) r0 = 0.f;
+    const float in[11] = {l0, l1, a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, r0};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int t = 0; t < 5; ++t) acc[j] = fmaf(in[2 * j + t], w[t], acc[j]);
+}
+
+template <bool VEC, int STRIDE>
+__global__ void __launch_bounds__(256)
+dw5_stream_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
+                  float* __restrict__ y, Status* status, uint32_t tag) {
+    const uint32_t tag_seen = __ldg(packed);
+    const float* __restrict__ wpk = reinterpret_cast<const float*>(packed + kHeaderBytes / 4);
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int sub = lane / c.XQ;
+    const int xq = lane - sub * c.XQ;
+    const uint32_t item = warp_global * (uint32_t)c.subs + (uint32_t)sub;
+    const bool live = (sub < c.subs) && (item < c.items);
+    uint32_t plane_idx = 0, chunk = 0;
+    c.div_chunks.divmod(live ? item : 0u, plane_idx, chunk);
+    const int ch = (int)(plane_idx % (uint32_t)s.C_in);
+    const float* __restrict__ xp = x + (size_t)plane_idx * s.H * s.W;
+    float* __restrict__ yp = y + (size_t)plane_idx * s.H_out * s.W_out;
+    const int col = xq * 4 * STRIDE;             // first input column of this strip
+    const int p0 = (int)chunk * c.RH;
+    const int p1 = min(p0 + c.RH, s.H_out);
+    const bool has_l = xq > 0, has_r = xq < c.XQ - 1;
+    const bool second_ok = STRIDE == 2 && col + 4 < s.W;
+    float w[5][5];
+#pragma unroll
+    for (int i = 0; i < 25; ++i) w[i / 5][i % 5] = live ? __ldg(wpk + (size_t)ch * 25 + i) : 0.f;
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // input rows STRIDE*p - 2 .. STRIDE*p + 2 feed output row p; STRIDE new rows per output row
+    float4 ra[5], rb[5], na[STRIDE], nb[STRIDE];
+#pragma unroll
+    for (int j = 0; j < 5; ++j) {
+        ra[j] = live ? ldrow<VEC>(xp, STRIDE * p0 - 2 + j, s.H, s.W, col) : z4;
+        rb[j] = (live && second_ok) ? ldrow<VEC>(xp, STRIDE * p0 - 2 + j, s.H, s.W, col + 4) : z4;
+    }
+    for (int p = p0; p < p0 + c.RH; ++p) {       // warp-uniform trip count
+#pragma unroll
+        for (int j = 0; j < STRIDE; ++j) {         // the next output row's new input rows, in flight during this row's math
+            const int h = STRIDE * (p + 1) + 3 - STRIDE + j;
+            const bool need = live && (p + 1 < p1);
+            na[j] = need ? ldrow<VEC>(xp, h, s.H, s.W, col) : z4;
+            nb[j] = (need && second_ok) ? ldrow<VEC>(xp, h, s.H, s.W, col + 4) : z4;
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int r = 0; r < 5; ++r) {
+            if constexpr (STRIDE == 1) row_taps5_s1(ra[r], has_l, has_r, w[r], acc);
+            else row_taps5_s2(ra[r], rb[r], has_l, has_r, w[r], acc);
+        }
+        if (live && p < p1 && tag_seen == tag) {
+            float* dst = yp + (size_t)p * s.W_out + xq * 4;
+            if ((s.W_out & 3) == 0) {
+                *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (xq * 4 + j < s.W_out) dst[j] = acc[j];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j + STRIDE < 5; ++j) { ra[j] = ra[j + STRIDE]; rb[j] = rb[j + STRIDE]; }
+#pragma unroll
+        for (int j = 0; j < STRIDE; ++j) { ra[5 - STRIDE + j] = na[j]; rb[5 - STRIDE + j] = nb[j]; }
+    }
+    if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
+}
+
 }  // namespace
 
 bool dw_supported(const Shape& s) {
-    if (!(s.KH == 3 && s.KW == 3 && s.dilation == 1 && s.pad == 1 && (s.stride == 1 || s.stride == 2))) return false;
+    const bool k3 = s.KH == 3 && s.KW == 3 && s.pad == 1, k5 = s.KH == 5 && s.KW == 5 && s.pad == 2;
+    if (!((k3 || k5) && s.dilation == 1 && (s.stride == 1 || s.stride == 2))) return false;
     if (!(s.Cg == 1 && s.Kg == 1)) return false;
     const int xq = s.stride == 1 ? (s.W + 3) / 4 : (s.W + 7) / 8;
     if (xq > 32) return false;
@@ -219,6 +314,16 @@ cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float
     const uint32_t tag = pack_tag(s, GCONV_VARIANT_DIRECT_TILED);
     const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed);
     const bool vec = (s.W % 4 == 0);
+    if (s.KH == 5) {
+        if (s.stride == 1) {
+            if (vec) dw5_stream_kernel<true, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+            else dw5_stream_kernel<false, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        } else {
+            if (vec) dw5_stream_kernel<true, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+            else dw5_stream_kernel<false, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        }
+        return cudaGetLastError();
+    }
     if (s.stride == 1) {
         if (vec) dw_stream_s1_kernel<true><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
         else dw_stream_s1_kernel<false><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);

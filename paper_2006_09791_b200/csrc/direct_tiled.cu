@@ -173,7 +173,8 @@ direct_tiled_kernel(const Shape s, const TiledCfg c, const float* __restrict__ x
 }
 
 __global__ void tiled_pack_kernel(Shape s, const float* __restrict__ w, uint32_t* __restrict__ packed, uint32_t tag) {
-    const size_t n = (size_t)s.C_out * s.Cg * 9;
+    const int taps = s.KH * s.KW;               // 9, or 25 for the 5x5 depthwise layers
+    const size_t n = (size_t)s.C_out * s.Cg * taps;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         packed[0] = tag;
@@ -181,14 +182,14 @@ __global__ void tiled_pack_kernel(Shape s, const float* __restrict__ w, uint32_t
     }
     float* dst = reinterpret_cast<float*>(packed + kHeaderBytes / 4);
     for (; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        // destination index i = (((g*Cg + c)*9 + rs)*Kg + k)
+        // destination index i = (((g*Cg + c)*taps + rs)*Kg + k)
         const int k = (int)(i % s.Kg);
         size_t t = i / s.Kg;
-        const int rs = (int)(t % 9);
-        t /= 9;
+        const int rs = (int)(t % taps);
+        t /= taps;
         const int c = (int)(t % s.Cg);
         const int g = (int)(t / s.Cg);
-        dst[i] = w[(((size_t)g * s.Kg + k) * s.Cg + c) * 9 + rs];
+        dst[i] = w[(((size_t)g * s.Kg + k) * s.Cg + c) * taps + rs];
     }
 }
 
@@ -202,13 +203,14 @@ int largest_kt(int Kg) {
 }  // namespace
 
 bool tiled_supported(const Shape& s) {
+    if (s.KH == 5 && s.KW == 5) return dw_supported(s);   // 5x5: only the depthwise stream kernel
     return s.KH == 3 && s.KW == 3 && s.dilation == 1 && (s.stride == 1 || s.stride == 2) && s.N <= 65535;
 }
 
-size_t tiled_packed_bytes(const Shape& s) { return kHeaderBytes + sizeof(float) * (size_t)s.C_out * s.Cg * 9; }
+size_t tiled_packed_bytes(const Shape& s) { return kHeaderBytes + sizeof(float) * (size_t)s.C_out * s.Cg * s.KH * s.KW; }
 
 cudaError_t tiled_pack(const Shape& s, const float* w, void* packed, cudaStream_t st) {
-    const size_t n = (size_t)s.C_out * s.Cg * 9;
+    const size_t n = (size_t)s.C_out * s.Cg * s.KH * s.KW;
     int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
     tiled_pack_kernel<<<blocks, 256, 0, st>>>(s, w, reinterpret_cast<uint32_t*>(packed), pack_tag(s, GCONV_VARIANT_DIRECT_TILED));
     return cudaGetLastError();

@@ -142,3 +142,10 @@ def mobilenetv2_dw_layers(N: int = 64) -> List[Layer]:
     mk = lambda C, HW, s: Layer("mbv2_dw_%d@%d%s" % (C, HW, "s2" if s == 2 else ""), N, C, HW, HW, C, stride=s, groups=C)
     return [mk(32, 112, 1), mk(96, 112, 2), mk(144, 56, 1), mk(144, 56, 2), mk(192, 28, 1), mk(192, 28, 2),
             mk(384, 14, 1), mk(576, 14, 1), mk(576, 14, 2), mk(960, 7, 1)]
+
+
+def depthwise5x5_layers(N: int = 64) -> List[Layer]:
+    """Depthwise 5x5 layers (pad 2, stride 1 and 2) at the sizes later mobile networks use them: 56x56 down to 7x7,
+    widths 72...960.  The second depthwise family of the follow-up items."""
+    mk = lambda C, HW, s: Layer("dw5_%d@%d%s" % (C, HW, "s2" if s == 2 else ""), N, C, HW, HW, C, 5, 5, s, 2, 1, C)
+    return [mk(72, 56, 2), mk(120, 28, 1), mk(240, 28, 2), mk(672, 14, 1), mk(672, 14, 2), mk(960, 7, 1)]

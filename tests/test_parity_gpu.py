@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
-from paper_2006_09791_b200.workloads import (Layer, config0, mobilenetv2_dw_layers, resnet34_layers, resnext_layers,
+from paper_2006_09791_b200.workloads import (Layer, config0, depthwise5x5_layers, mobilenetv2_dw_layers, resnet34_layers, resnext_layers,
                                              sweep_layers, wrn_stack)
 
 from golden_io import load_case
@@ -161,6 +161,27 @@ def _seeded_random_shapes(seed, count):
 def test_seeded_random_shapes(chunk):
     for i, cfg in enumerate(_seeded_random_shapes(20260 + chunk, 25)):
         check_layer(Layer("rand%d_%d" % (chunk, i), *cfg), seed=100 * chunk + i)
+
+
+DW5_SHAPES = [
+    # N, C, H, W, C_out, 5, 5, stride, pad 2, dilation 1, groups = C: widths around the 4- and 8-column strips, odd sizes
+    (2, 8, 9, 7, 8, 5, 5, 1, 2, 1, 8), (1, 5, 13, 13, 5, 5, 5, 2, 2, 1, 5), (3, 16, 20, 24, 16, 5, 5, 1, 2, 1, 16),
+    (2, 12, 17, 33, 12, 5, 5, 2, 2, 1, 12), (1, 4, 6, 128, 4, 5, 5, 1, 2, 1, 4), (2, 6, 5, 5, 6, 5, 5, 1, 2, 1, 6),
+    (1, 3, 31, 64, 3, 5, 5, 2, 2, 1, 3), (2, 10, 12, 10, 10, 5, 5, 2, 2, 1, 10), (1, 7, 40, 36, 7, 5, 5, 1, 2, 1, 7),
+]
+
+
+@pytest.mark.parametrize("cfg", DW5_SHAPES)
+def test_depthwise_5x5_shapes(cfg):
+    L = Layer("dw5", *cfg)
+    err, used = check_layer(L, seed=5)
+    assert used == gconv.GCONV_VARIANT_DIRECT_TILED           # the stream kernel, not the generic fallback
+    check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=5)
+
+
+def test_depthwise_5x5_network_shapes():
+    for L in depthwise5x5_layers(N=2):
+        check_layer(L)
 
 
 def test_pack_mismatch_is_reported_not_fatal():
