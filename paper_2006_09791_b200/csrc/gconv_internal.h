@@ -123,6 +123,7 @@ struct IgemmCfg {
     int issuers;             // MMA-issuing warps (2 or 4), one per accumulator buffer
     int egroups, threads;    // epilogue groups of eight warps (1 or 2) and the block size that goes with them
     int cps;                 // CTAs per (group, filter tile) when the grid is split into one set per pair, else 0
+    int tapb;                // one stage holds three blocks of four segments, one per vertical tap (small planes)
     int tmem_cols;           // TMEM columns the CTA allocates (power of two >= nacc * Np)
     uint32_t xchg_off;       // offset of the edge-lane exchange area in dynamic shared memory
     int fast4;               // a second tensor map for whole-tile copies is available

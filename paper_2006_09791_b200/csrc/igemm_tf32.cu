@@ -190,25 +190,26 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4;
+        nt_fast, wseg, nseg, SR, fast4, tapb;
 };
-constexpr int kFamilies = 10;
+constexpr int kFamilies = 11;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  1}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9,  1,  1}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4,  0, -1}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1}     // row boxes of one segment, narrow groups
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  1,  0}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9,  1,  1,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0}     // row boxes of one segment, narrow groups
+         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -377,7 +378,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 if (!box) {
                     if (!have_lane_coords) {
                         uint32_t n, i;
-                        if (c.nr == 3) {                   // tile plus halo: contiguous segments of one image
+                        if (c.tapb) {                      // lane = 4 * tap + segment: the tap's own row shift, any image
+                            c.div_spi.divmod(mt * 4u + (uint32_t)(lane & 3), n, i);
+                            my_n = (int)n < s.N ? (int)n : s.N;
+                            my_f = (int)i * 32 + ((lane >> 2) - 1) * s.W;
+                        } else if (c.nr == 3) {            // tile plus halo: contiguous segments of one image
                             c.div_spi.divmod(c.seg_mode ? mt * 4u : mt, n, i);
                             my_n = (int)n;
                             my_f = (c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W) + (lane - c.wseg) * 32;
@@ -868,6 +873,18 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
     }
+    // Tap blocks: small planes whose rows are shorter than a segment (16x16, 8x8) cannot take the taps as views of one
+    // halo block, but narrow groups can still stage all three taps of a tile in ONE stage -- three blocks of four
+    // segments, each loaded with its own row shift -- so a tile costs one barrier round trip instead of three.  Only
+    // where a tile straddles images anyway (8x8): 16x16 planes keep their one-box-per-tap copies, which are faster.
+    c.tapb = 0;
+    if (c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
+        3u * (uint32_t)c.Cg * (uint32_t)c.Np * 4u <= 40u * 1024u) {
+        c.tapb = 1;
+        c.nr = 3;
+        c.wseg = 4;
+        c.nseg = 12;
+    }
     c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.issuers = c.nacc;                                // MMA-issuing warps: one per accumulator buffer
@@ -904,7 +921,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
         const uint32_t st_bytes = (a_bytes + 1023u) & ~1023u;
         const int kst = (3 / c.nr) * c.chunks;
         const bool fits = 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
-                          c.bres_stride + (uint32_t)(kst == 1 ? 2 : kst + 1) * st_bytes + xchg_bytes + 1024u <= light_total;
+                          c.bres_stride + (uint32_t)(c.tapb ? 1 : (kst == 1 ? 2 : kst + 1)) * st_bytes + xchg_bytes + 1024u <= light_total;
         if (fits) {
             c.b_res = 1;
             c.nacc = 2;
@@ -920,7 +937,8 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     const uint32_t budget = budget_total - (uint32_t)c.b_res * c.bres_stride - xchg_bytes;
     int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
-    if (st < 2) st = 2;
+    if (st < 2 && !c.tapb) st = 2;
+    if (st < 1) st = 1;
     c.stages = st;
     c.xchg_off = (uint32_t)c.stages * c.stage_bytes + (uint32_t)c.b_res * c.bres_stride;
     c.smem_bytes = (size_t)c.xchg_off + xchg_bytes + 1024;
@@ -1001,7 +1019,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
         cfg.fast4 = 1;   // the second map is in use (prefetch it)
-    } else if (c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
+    } else if (!c.tapb && c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
         const cuuint64_t dims4[4] = {HW, (cuuint64_t)s.C_in, 8, (cuuint64_t)s.N};
         const cuuint64_t strides4[3] = {HW * 4, 128, HW * 4 * (cuuint64_t)s.C_in};
         const cuuint32_t box4[4] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.nseg, 1};
@@ -1017,7 +1035,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     static const KernelFn kernels[kFamilies] = {igemm_tf32_kernel<0>, igemm_tf32_kernel<1>, igemm_tf32_kernel<2>,
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
-                                                igemm_tf32_kernel<9>};
+                                                igemm_tf32_kernel<9>, igemm_tf32_kernel<10>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
