@@ -196,7 +196,7 @@ constexpr int kFamilies = 11;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  1,  0}     // 32-wide planes with halo stages
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0}     // 32-wide planes with halo stages
          : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0}     // row boxes of two segments, narrow groups
          : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9,  1,  1,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
          : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0}     // stride-2 row tiles, narrow groups
@@ -366,11 +366,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
                 const int chan = g * c.Cg + ch * c.CK;
                 const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
-                const bool box = c.rowbox || (c.fast4 && lo >= 0 && lo + c.nseg * 32 <= HW);
+                const bool box = c.rowbox || c.fast4 == 2 || (c.fast4 == 1 && lo >= 0 && lo + c.nseg * 32 <= HW);
                 if (lane == 0) {
                     mbar_arrive_expect_tx(full, a_bytes + nb);
                     if (box) {
                         if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, rb_seg, rb_row0, tile_n, full);   // rows above/below and columns past W: zero fill
+                        else if (c.fast4 == 2) tma_load_4d(a_dst, &xmap4, 0, chan, lo >> 5, tile_n, full);   // segments outside the plane read as zeros
                         else tma_load_4d(a_dst, &xmap4, lo, chan, 0, tile_n, full);
                     }
                     if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
@@ -1019,6 +1020,20 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
         cfg.fast4 = 1;   // the second map is in use (prefetch it)
+    } else if (c.nr == 3 && !c.tapb && HW % 32 == 0) {
+        // Halo stages of segment or flat-row tiles: (pixel in segment, channel, segment of the plane, image).  The box
+        // starts wseg segments before the tile; segments before or after the plane are out of range and read as zeros,
+        // so the first and last tiles of a plane are whole boxes too.
+        const cuuint64_t dims4[4] = {32, (cuuint64_t)s.C_in, HW / 32, (cuuint64_t)s.N};
+        const cuuint64_t strides4[3] = {HW * 4, 128, HW * 4 * (cuuint64_t)s.C_in};
+        const cuuint32_t box4[4] = {32, (cuuint32_t)c.CK, (cuuint32_t)c.nseg, 1};
+        const cuuint32_t estr4[4] = {1, 1, 1, 1};
+        if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims4, strides4, box4, estr4,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+            cfg.fast4 = 2;
+        else
+            xmap4 = xmap;
     } else if (!c.tapb && c.seg_fstep == 32 && (!c.seg_mode || c.SPI % 4 == 0)) {
         const cuuint64_t dims4[4] = {HW, (cuuint64_t)s.C_in, 8, (cuuint64_t)s.N};
         const cuuint64_t strides4[3] = {HW * 4, 128, HW * 4 * (cuuint64_t)s.C_in};
