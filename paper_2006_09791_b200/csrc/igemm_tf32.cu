@@ -47,6 +47,7 @@ constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issu
 constexpr int kThreads = 32 * (kMmaWarp3 + 2);
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
+constexpr uint32_t kPrefetchUses = 1;   // stages whose input is prefetched into L2 before the dependency wait
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr int kMaxDynSmem = 226 * 1024;   // 227 KB per CTA minus the static control block (under 1 KB)
 
@@ -123,6 +124,19 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
         : "memory");
+}
+// L2 prefetch of the same boxes (a cache hint: nothing is written, no barrier is involved)
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2),
+                 "r"(c3), "r"(c4)
+                 : "memory");
 }
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -329,15 +343,28 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             cur_gn = (int)gn;
             switches = 1;
         }
-        asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
-        for (int tile = tile_first; tile < tile_end && ok; tile += tile_step) {
+        // Two passes over the tiles.  Pass 0 runs before the dependency wait and only asks L2 to fetch the input box of
+        // the first stage: a cache hint, nothing is consumed, and L2 is the point of coherence, so it stays correct if
+        // the previous kernel is still writing those lines (then they are in L2 already).  The CTA usually sits in the
+        // wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2 instead
+        // of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
+        // Pass 1 is the real one.
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+        const bool pf = pass == 0;
+        if (!pf) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
+            it = 0;
+            stage = 0;
+            ph = 0;
+        }
+        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile += tile_step) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
             uint32_t gq = gn, ntq = 0;
             if (c.NT > 1) c.div_nt.divmod(gn, gq, ntq);
             const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
-            const bool switch_b = c.b_res && (int)gn != cur_gn;
+            const bool switch_b = !pf && c.b_res && (int)gn != cur_gn;
             // Whole-tile copies: a row-box tile is always one 5-D box; a flat tile whose segments are one contiguous run
             // is one 4-D box for every tap whose run stays inside the image plane.  Everything else (tiles that straddle
             // images, and the plane's first/last tiles, whose out-of-plane part must be zero-filled) is copied segment
@@ -359,15 +386,22 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             bool have_lane_coords = false;
             int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
+                if (pf && it >= kPrefetchUses) break;
                 // the first pass over the ring finds every stage free
-                if (it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                if (!pf && it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
                 const int chan = g * c.Cg + ch * c.CK;
                 const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
                 const bool box = c.rowbox || c.fast4 == 2 || (c.fast4 == 1 && lo >= 0 && lo + c.nseg * 32 <= HW);
-                if (lane == 0) {
+                if (lane == 0 && pf) {
+                    if (box) {
+                        if (c.rowbox) tma_prefetch_5d(&xmap4, 0, chan, rb_seg, rb_row0, tile_n);
+                        else if (c.fast4 == 2) tma_prefetch_4d(&xmap4, 0, chan, lo >> 5, tile_n);
+                        else tma_prefetch_4d(&xmap4, lo, chan, 0, tile_n);
+                    }
+                } else if (lane == 0) {
                     mbar_arrive_expect_tx(full, a_bytes + nb);
                     if (box) {
                         if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, rb_seg, rb_row0, tile_n, full);   // rows above/below and columns past W: zero fill
@@ -399,7 +433,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         have_lane_coords = true;
                     }
                     __syncwarp();                          // the barrier is armed before any lane's copy can complete on it
-                    if (lane < c.nseg) tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, chan, my_n, full);
+                    if (lane < c.nseg) {
+                        if (pf) tma_prefetch_3d(&xmap, my_f + (r - 1) * s.W, chan, my_n);
+                        else tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, chan, my_n, full);
+                    }
                 }
                 if (ks == 0 && switch_b) {
                     // New (group, filter tile): its weights go to the free resident buffer.  Issued after the tile's
@@ -417,6 +454,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
+        }
         }
         if (!ok && lane == 0) {
             // drain: wait (bounded) for the copies of every stage that may still be in flight
