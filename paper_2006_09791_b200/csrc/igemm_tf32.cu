@@ -212,11 +212,11 @@ __host__ __device__ constexpr Family family(int f) {
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, narrow groups
          : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0}     // 32-wide planes with halo stages
          : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2,  0, -1,  1,   9,  1,  1,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
          : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0}     // stride-2 row tiles, narrow groups
          : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, streamed weights
          : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2,  0, -1,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
          : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0}     // row boxes of one segment, narrow groups
          : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1}     // 16x16 / 8x8 planes, narrow groups, tap blocks
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1};
