@@ -22,13 +22,18 @@
 //     tcgen05.ld, apply the horizontal shifts with warp shuffles and write y directly in NCHW with
 //     128-byte coalesced rows.
 // Stride 2 (pad 1) keeps the even rows and columns of that stride-1 result: same operands, the
-// epilogue stores only those lanes (and for W = 32 the odd rows are never loaded or multiplied).
+// epilogue stores only those lanes; for widths 16..62 a tile is four OUTPUT rows and the odd input rows are never
+// multiplied (their stage holds nine input rows, a tap is the view of every other one).
 // All groups and all images run in one persistent launch: the tile index enumerates
-// (group, filter tile, pixel tile), one CTA per SM walks it.
+// (group, filter tile, pixel tile).  Two launch shapes: one CTA per SM with all 21 warps ("heavy"), or two CTAs per SM
+// of 11 warps each ("light": small filter banks, two accumulators in 256 TMEM columns, half the shared memory).
+// The kernel body is written once against the run-time configuration and compiled in a few "families" whose mode
+// fields are compile-time constants (see Family below); the host picks the instantiation.
 //
 // Warp roles: warp 0 = TMA producer, warps 1, 10 (and 19, 20 when four accumulators fit) = single-thread MMA issuers
 // taking tiles in turn, each with its own accumulator buffer (warp 1 owns the TMEM allocation),
-// warps 2..9 and 11..18 = two epilogue groups for alternate tiles (TMEM lane quarter = warp_id % 4).
+// warps 2..9 and 11..18 = two epilogue groups for alternate tiles (TMEM lane quarter = warp_id % 4); the light shape
+// launches warps 0..10 only.
 // Every mbarrier wait is bounded: when a
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
 // copies are waited for (bounded), TMEM is freed and the kernel returns.
