@@ -10,7 +10,8 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
-from paper_2006_09791_b200.workloads import sweep_layers, wrn_stack
+from paper_2006_09791_b200.workloads import (depthwise5x5_layers, mobilenetv2_dw_layers, resnext_layers, sweep_layers,
+                                             wrn_stack)
 
 pytestmark = pytest.mark.gpu
 
@@ -82,6 +83,20 @@ def test_group_sweep_at_batch_32(idx):
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(78, idx), L.x_dist)
     y, v = _run_full(L, x, w, use_graph=True)
     _check_samples(L, y, x, w, v, _samples(L, 3 if L.groups == 1 else 6, idx))
+
+
+def _sweep_row_families():
+    """The other rows of the bench's sweep table at the batch it times them at: ResNeXt-shaped grouped layers (stride-2
+    row tiles, padded 14x14 and 7x7 planes, tap blocks), MobileNetV2-shaped depthwise 3x3 and depthwise 5x5 layers."""
+    return resnext_layers(64) + mobilenetv2_dw_layers(64)[4:] + depthwise5x5_layers(64)[1:]
+
+
+@pytest.mark.parametrize("idx", range(len(_sweep_row_families())))
+def test_sweep_table_rows_at_batch_64(idx):
+    L = _sweep_row_families()[idx]
+    x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.groups, synth.layer_seed(80, idx), L.x_dist)
+    y, v = _run_full(L, x, w, use_graph=(idx % 2 == 1))
+    _check_samples(L, y, x, w, v, _samples(L, 6, idx))
 
 
 def test_more_than_2_to_31_elements():
