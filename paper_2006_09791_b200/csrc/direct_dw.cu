@@ -16,14 +16,19 @@ namespace {
 
 constexpr int U = 4;   // output rows per pipeline block
 
-// Four consecutive pixels of row h starting at column col (zero outside the image).  VEC: W % 4 == 0, so the
-// address is 16-byte aligned and the four pixels are in range; otherwise four bounds-checked scalar loads.
-template <bool VEC>
+// Four consecutive pixels of row h starting at column col (zero outside the image).  VEC = 4: W % 4 == 0, so the
+// address is 16-byte aligned and the four pixels are in range; VEC = 2: W is even, two 8-byte loads (the second pair
+// may be past the row); VEC = 0: four bounds-checked scalar loads.
+template <int VEC>
 __device__ __forceinline__ float4 ldrow(const float* __restrict__ plane, int h, int H, int W, int col) {
     if (h < 0 || h >= H) return make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = plane + (size_t)h * W + col;
-    if constexpr (VEC) {
+    if constexpr (VEC == 4) {
         return __ldg(reinterpret_cast<const float4*>(p));
+    } else if constexpr (VEC == 2) {
+        const float2 a = __ldg(reinterpret_cast<const float2*>(p));
+        const float2 b = col + 2 < W ? __ldg(reinterpret_cast<const float2*>(p + 2)) : make_float2(0.f, 0.f);
+        return make_float4(a.x, a.y, b.x, b.y);
     } else {
         float4 v;
         v.x = col + 0 < W ? __ldg(p + 0) : 0.f;
@@ -33,10 +38,13 @@ __device__ __forceinline__ float4 ldrow(const float* __restrict__ plane, int h, 
         return v;
     }
 }
-template <bool VEC>
+template <int VEC>
 __device__ __forceinline__ void strow(float* __restrict__ dst, int col, int W, const float (&acc)[4]) {
-    if constexpr (VEC) {
+    if constexpr (VEC == 4) {
         *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    } else if constexpr (VEC == 2) {
+        *reinterpret_cast<float2*>(dst) = make_float2(acc[0], acc[1]);
+        if (col + 2 < W) *reinterpret_cast<float2*>(dst + 2) = make_float2(acc[2], acc[3]);
     } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j)
@@ -56,7 +64,7 @@ __device__ __forceinline__ void row_taps1(const float4 v, bool has_l, bool has_r
     acc[3] = fmaf(v.z, w[0], acc[3]); acc[3] = fmaf(v.w, w[1], acc[3]); acc[3] = fmaf(r, w[2], acc[3]);
 }
 
-template <bool VEC>
+template <int VEC>
 __global__ void __launch_bounds__(256)
 dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
@@ -119,7 +127,7 @@ __device__ __forceinline__ void row_taps2(const float4 a, const float4 b, bool h
     acc[3] = fmaf(b.y, w[0], acc[3]); acc[3] = fmaf(b.z, w[1], acc[3]); acc[3] = fmaf(b.w, w[2], acc[3]);
 }
 
-template <bool VEC>
+template <int VEC>
 __global__ void __launch_bounds__(256)
 dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
@@ -170,6 +178,9 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
             float* dst = yp + (size_t)p * s.W_out + xq * 4;
             if ((s.W_out & 3) == 0) {
                 *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else if ((s.W_out & 1) == 0) {
+                *reinterpret_cast<float2*>(dst) = make_float2(acc[0], acc[1]);
+                if (xq * 4 + 2 < s.W_out) *reinterpret_cast<float2*>(dst + 2) = make_float2(acc[2], acc[3]);
             } else {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -213,7 +224,7 @@ __device__ __forceinline__ void row_taps5_s2(const float4 a, const float4 b, boo
         for (int t = 0; t < 5; ++t) acc[j] = fmaf(in[2 * j + t], w[t], acc[j]);
 }
 
-template <bool VEC, int STRIDE>
+template <int VEC, int STRIDE>
 __global__ void __launch_bounds__(256)
 dw5_stream_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                   float* __restrict__ y, Status* status, uint32_t tag) {
@@ -264,6 +275,9 @@ dw5_stream_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, con
             float* dst = yp + (size_t)p * s.W_out + xq * 4;
             if ((s.W_out & 3) == 0) {
                 *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            } else if ((s.W_out & 1) == 0) {
+                *reinterpret_cast<float2*>(dst) = make_float2(acc[0], acc[1]);
+                if (xq * 4 + 2 < s.W_out) *reinterpret_cast<float2*>(dst + 2) = make_float2(acc[2], acc[3]);
             } else {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -313,24 +327,28 @@ cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float
     const DwCfg c = dw_config(s, sm_count);
     const uint32_t tag = pack_tag(s, GCONV_VARIANT_DIRECT_TILED);
     const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed);
-    const bool vec = (s.W % 4 == 0);
+    const int vec = s.W % 4 == 0 ? 4 : (s.W % 2 == 0 ? 2 : 0);
+#define GCONV_DW_LAUNCH(KERNEL) \
+    do { \
+        if (vec == 4) KERNEL(4); else if (vec == 2) KERNEL(2); else KERNEL(0); \
+    } while (0)
+#define GCONV_DW5_S1(V) dw5_stream_kernel<V, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
+#define GCONV_DW5_S2(V) dw5_stream_kernel<V, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
+#define GCONV_DW3_S1(V) dw_stream_s1_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
+#define GCONV_DW3_S2(V) dw_stream_s2_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
     if (s.KH == 5) {
-        if (s.stride == 1) {
-            if (vec) dw5_stream_kernel<true, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-            else dw5_stream_kernel<false, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-        } else {
-            if (vec) dw5_stream_kernel<true, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-            else dw5_stream_kernel<false, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-        }
-        return cudaGetLastError();
-    }
-    if (s.stride == 1) {
-        if (vec) dw_stream_s1_kernel<true><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-        else dw_stream_s1_kernel<false><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        if (s.stride == 1) GCONV_DW_LAUNCH(GCONV_DW5_S1);
+        else GCONV_DW_LAUNCH(GCONV_DW5_S2);
+    } else if (s.stride == 1) {
+        GCONV_DW_LAUNCH(GCONV_DW3_S1);
     } else {
-        if (vec) dw_stream_s2_kernel<true><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
-        else dw_stream_s2_kernel<false><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag);
+        GCONV_DW_LAUNCH(GCONV_DW3_S2);
     }
+#undef GCONV_DW_LAUNCH
+#undef GCONV_DW5_S1
+#undef GCONV_DW5_S2
+#undef GCONV_DW3_S1
+#undef GCONV_DW3_S2
     return cudaGetLastError();
 }
 
