@@ -790,9 +790,14 @@ __global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict_
         float v[4] = {0.f, 0.f, 0.f, 0.f};
         if (h < H) {
             const float* src = x + (plane * H + h) * (size_t)W;
+            if ((W & 1) == 0) {                    // even width: rows start on 8-byte boundaries
+                if (w4 < W) { const float2 a = __ldg(reinterpret_cast<const float2*>(src + w4)); v[0] = a.x; v[1] = a.y; }
+                if (w4 + 2 < W) { const float2 b = __ldg(reinterpret_cast<const float2*>(src + w4 + 2)); v[2] = b.x; v[3] = b.y; }
+            } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (w4 + j < W) v[j] = __ldg(src + w4 + j);
+                for (int j = 0; j < 4; ++j)
+                    if (w4 + j < W) v[j] = __ldg(src + w4 + j);
+            }
         }
         *reinterpret_cast<float4*>(xp + (plane * Hp + h) * (size_t)Wp + w4) = make_float4(v[0], v[1], v[2], v[3]);
     }
