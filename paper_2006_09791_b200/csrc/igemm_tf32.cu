@@ -780,13 +780,30 @@ static IgemmGeom igemm_geom(const Shape& s) {
 }
 
 namespace {
-__global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict__ xp, size_t planes, int H, int W, int Hp, int Wp) {
+// Zero-padded copy of x for widths TMA cannot address: every plane becomes Hp x Wp (Wp a multiple of 4), one thread
+// per group of four output columns.  IDX is the index type: 32-bit whenever the padded tensor has fewer than 2^32
+// column groups (the common case: the divisions are then cheap multiply-shift ones).
+template <typename IDX>
+__global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict__ xp, size_t planes, int H, int W, int Hp, int Wp,
+                                 FastDiv div_plane, FastDiv div_row) {
     const size_t per_plane = (size_t)Hp * (Wp / 4);
     const size_t total = planes * per_plane;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const size_t plane = i / per_plane;
-        const int rem = (int)(i - plane * per_plane);
-        const int h = rem / (Wp / 4), w4 = (rem - h * (Wp / 4)) * 4;
+        size_t plane;
+        int h, w4;
+        if constexpr (sizeof(IDX) == 4) {
+            uint32_t pl, rem, hh, q;
+            div_plane.divmod((uint32_t)i, pl, rem);
+            div_row.divmod(rem, hh, q);
+            plane = pl;
+            h = (int)hh;
+            w4 = (int)q * 4;
+        } else {
+            plane = i / per_plane;
+            const int rem = (int)(i - plane * per_plane);
+            h = rem / (Wp / 4);
+            w4 = (rem - h * (Wp / 4)) * 4;
+        }
         float v[4] = {0.f, 0.f, 0.f, 0.f};
         if (h < H) {
             const float* src = x + (plane * H + h) * (size_t)W;
@@ -1032,7 +1049,11 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
         const size_t planes = (size_t)s.N * s.C_in;
         const size_t total = planes * ge.Hp * (ge.Wp / 4);
         const int blocks = (int)((total + 255) / 256 < (size_t)sm_count * 16 ? (total + 255) / 256 : (size_t)sm_count * 16);
-        igemm_pad_kernel<<<blocks, 256, 0, st>>>(x_in, scratch, planes, s.H, s.W, ge.Hp, ge.Wp);
+        const FastDiv div_plane = make_fastdiv((uint32_t)(ge.Hp * (ge.Wp / 4))), div_row = make_fastdiv((uint32_t)(ge.Wp / 4));
+        if (total < (1ull << 32))
+            igemm_pad_kernel<uint32_t><<<blocks, 256, 0, st>>>(x_in, scratch, planes, s.H, s.W, ge.Hp, ge.Wp, div_plane, div_row);
+        else
+            igemm_pad_kernel<uint64_t><<<blocks, 256, 0, st>>>(x_in, scratch, planes, s.H, s.W, ge.Hp, ge.Wp, div_plane, div_row);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         s.H = ge.Hp;
