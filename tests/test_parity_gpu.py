@@ -184,6 +184,64 @@ def test_depthwise_5x5_network_shapes():
         check_layer(L)
 
 
+@pytest.mark.parametrize("shape", [(16, 32, 32, 32, 4), (8, 64, 16, 16, 2), (24, 128, 8, 8, 8), (6, 64, 28, 28, 1), (4, 16, 56, 56, 16),
+                                   (4, 32, 14, 14, 4), (8, 32, 28, 28, 32), (3, 256, 14, 14, 1)])
+def test_dependent_chain_back_to_back(shape):
+    """Five layers launched back to back on one stream, each reading the previous layer's output (the kernels start
+    their set-up, weight fetch and an L2 prefetch before the previous kernel has finished, so this is the case that
+    must not read early): once eagerly and once as a CUDA-graph replay over NaN-filled buffers.  Every layer's output
+    is compared with the oracle applied to the input that layer actually saw on the GPU."""
+    N, C, H, W, groups = shape
+    L = Layer("chain", N, C, H, W, C, groups=groups)
+    dev = torch.device("cuda:0")
+    depth = 5
+    x0, _ = synth.make_layer_tensors(N, C, H, W, C, 3, 3, groups, synth.layer_seed(31, N, C, groups))
+    ws = [synth.make_layer_tensors(1, C, H, W, C, 3, 3, groups, synth.layer_seed(32, k, C, groups))[1] for k in range(depth)]
+    descs = [gconv.gconv_desc_create(*L.desc_args()) for _ in range(depth)]
+    try:
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            bufs = [torch.from_numpy(x0).to(dev)] + [torch.empty(L.y_elems, dtype=torch.float32, device=dev) for _ in range(depth)]
+            wps = []
+            for d, w in zip(descs, ws):
+                wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+                gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp, stream)
+                wps.append(wp)
+
+            def run_chain():
+                for k in range(depth):
+                    gconv.gconv_forward(descs[k], bufs[k], wps[k], bufs[k + 1], stream)
+
+            for use_graph in (False, True):
+                for b in bufs[1:]:
+                    b.fill_(float("nan"))
+                if use_graph:
+                    run_chain()                      # (descriptor-owned allocations happen outside the capture)
+                    stream.synchronize()
+                    for b in bufs[1:]:
+                        b.fill_(float("nan"))
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=stream):
+                        run_chain()
+                    for b in bufs[1:]:
+                        b.fill_(float("nan"))
+                    graph.replay()
+                else:
+                    run_chain()
+                stream.synchronize()
+                for d in descs:
+                    assert gconv.gconv_last_status(d, stream) == gconv.GCONV_OK
+                outs = [bufs[0].cpu().numpy()] + [b.cpu().numpy().reshape(N, C, H, W) for b in bufs[1:]]
+                for k in range(depth):
+                    assert np.all(np.isfinite(outs[k + 1])), "layer %d wrote a non-finite value or skipped one" % k
+                    ref = oracle.gconv_ref(outs[k].reshape(N, C, H, W), ws[k], 1, 1, 1, groups, threads=8)
+                    err = rel_err(outs[k + 1], ref)
+                    assert err <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(descs[k])], (k, use_graph, err)
+    finally:
+        for d in descs:
+            gconv.gconv_desc_destroy(d)
+
+
 def test_pack_mismatch_is_reported_not_fatal():
     (L,) = config0()
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 5)
