@@ -170,6 +170,34 @@ int gconv_forward_host(gconv_desc_t desc, const float *x_host, const void *w_pac
  */
 int gconv_forward_host_static(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host, void *stream);
 
+/*
+ * Fused block: the grouped 3x3 convolution of the descriptor followed by a pointwise (1x1, groups = 1, no bias)
+ * convolution C_out -> C2, the block that replaces a standard convolution in Section II of the paper ("G(g)": a
+ * grouped convolution followed by a pointwise one that re-mixes the channels).  One kernel: the grouped result of a
+ * 128-pixel tile never leaves the SM (TMEM -> shared memory -> second tensor-core contraction), so x is read once
+ * and only y2 is written.  Runs on the tensor-core variant whatever variant the descriptor resolved to.
+ *
+ *   y2[n, k2, p, q] = sum_{o < C_out} w2[k2, o] * y[n, o, p, q],   y = the descriptor's grouped convolution of x
+ *
+ * gconv_block_supported  1 if the pair (descriptor, C2) can run fused, else 0: 3x3, pad 1, stride 1, dilation 1,
+ *                        W a multiple of 4 and at most 62 or equal to 64 wide planes only where the grouped kernel
+ *                        needs no edge exchange, merged group width a multiple of 8 with at most 64 filters per
+ *                        group, C2 a multiple of 16 with 2 * 3 * (filters per merged group) + C2 <= 512, and the
+ *                        resident pointwise weights (C_out * C2 * 4 bytes) must leave room for two input stages.
+ * gconv_block_packed_bytes  size of the packed buffer holding both weight tensors (0 if unsupported).
+ * gconv_block_pack_weights  w_ochw device fp32 [C_out, C_in/groups, 3, 3]; w2 device fp32 [C2, C_out]; both rounded
+ *                        to TF32 while packing; asynchronous on `stream`.
+ * gconv_block_forward    x device fp32 [N, C_in, H, W]; y2 device fp32 [N, C2, H_out, W_out]; asynchronous on
+ *                        `stream`; both TF32 contractions accumulate in FP32, the intermediate is kept in FP32 and
+ *                        consumed as TF32.  Tolerance: max|y2 - ref| / max|ref| <= 5e-3 against the oracle's grouped
+ *                        convolution followed by its 1x1 convolution.
+ * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_UNSUPPORTED, GCONV_ERR_CUDA; device status as gconv_forward.
+ */
+int gconv_block_supported(gconv_desc_t desc, int C2);
+size_t gconv_block_packed_bytes(gconv_desc_t desc, int C2);
+int gconv_block_pack_weights(gconv_desc_t desc, int C2, const float *w_ochw, const float *w2, void *w_packed, void *stream);
+int gconv_block_forward(gconv_desc_t desc, int C2, const float *x, const void *w_packed, float *y2, void *stream);
+
 /* Number of kernel launches one gconv_forward of this descriptor enqueues (for launch accounting). */
 int gconv_forward_launches(gconv_desc_t desc);
 

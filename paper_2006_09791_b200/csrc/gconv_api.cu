@@ -226,6 +226,32 @@ int gconv_forward_host(gconv_desc_t d, const float* x_host, const void* w_packed
     return GCONV_OK;
 }
 
+int gconv_block_supported(gconv_desc_t d, int C2) { return (d != nullptr && igemm_block_supported(d->s, C2)) ? 1 : 0; }
+
+size_t gconv_block_packed_bytes(gconv_desc_t d, int C2) {
+    return (d != nullptr && igemm_block_supported(d->s, C2)) ? igemm_block_packed_bytes(d->s, C2) : 0;
+}
+
+int gconv_block_pack_weights(gconv_desc_t d, int C2, const float* w_ochw, const float* w2, void* w_packed, void* stream) {
+    if (d == nullptr || w_ochw == nullptr || w2 == nullptr || w_packed == nullptr) return GCONV_ERR_NULL;
+    if (!aligned16(w_ochw) || !aligned16(w2) || !aligned16(w_packed)) return GCONV_ERR_ALIGNMENT;
+    if (!igemm_block_supported(d->s, C2)) return GCONV_ERR_UNSUPPORTED;
+    int rc = ensure_device_state(d);
+    if (rc != GCONV_OK) return rc;
+    const cudaError_t e = igemm_block_pack(d->s, C2, w_ochw, w2, w_packed, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GCONV_OK : fail_cuda(d, e);
+}
+
+int gconv_block_forward(gconv_desc_t d, int C2, const float* x, const void* w_packed, float* y2, void* stream) {
+    if (d == nullptr || x == nullptr || w_packed == nullptr || y2 == nullptr) return GCONV_ERR_NULL;
+    if (!aligned16(x) || !aligned16(w_packed) || !aligned16(y2)) return GCONV_ERR_ALIGNMENT;
+    if (!igemm_block_supported(d->s, C2)) return GCONV_ERR_UNSUPPORTED;
+    int rc = ensure_device_state(d);
+    if (rc != GCONV_OK) return rc;
+    const cudaError_t e = igemm_block_forward(d->s, C2, x, w_packed, y2, d->status_dev, d->sm_count, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GCONV_OK : fail_cuda(d, e);
+}
+
 int gconv_forward_launches(gconv_desc_t d) {
     if (d == nullptr) return 0;
     return (d->variant == GCONV_VARIANT_IGEMM_TF32 && igemm_scratch_bytes(d->s) > 0) ? 2 : 1;

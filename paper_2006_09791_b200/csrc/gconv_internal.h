@@ -124,6 +124,11 @@ struct IgemmCfg {
     int egroups, threads;    // epilogue groups of eight warps (1 or 2) and the block size that goes with them
     int cps;                 // CTAs per (group, filter tile) when the grid is split into one set per pair, else 0
     int tapb;                // one stage holds three blocks of four segments, one per vertical tap (small planes)
+    // fused grouped + pointwise block (0 for the plain convolution)
+    int fuse, C2, n_gn, d2_col;   // pointwise output channels, (group, filter tile) pairs per pixel tile, TMEM column of its accumulator
+    uint32_t w2_off, a2_off;      // shared-memory offsets of the resident pointwise weights and of the two A2 buffers
+    size_t w2_goff;               // byte offset of the pointwise weight blocks inside the packed buffer
+    FastDiv div_ngn;
     int tmem_cols;           // TMEM columns the CTA allocates (power of two >= nacc * Np)
     uint32_t xchg_off;       // offset of the edge-lane exchange area in dynamic shared memory
     int fast4;               // a second tensor map for whole-tile copies is available
@@ -140,6 +145,12 @@ bool igemm_supported(const Shape& s);
 IgemmCfg igemm_config(const Shape& s, int sm_count);
 size_t igemm_packed_bytes(const Shape& s);
 cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_t st);
+// fused block: grouped 3x3 (this shape) followed by a pointwise convolution C_out -> C2, one kernel, no intermediate in HBM
+bool igemm_block_supported(const Shape& s, int C2);
+size_t igemm_block_packed_bytes(const Shape& s, int C2);
+cudaError_t igemm_block_pack(const Shape& s, int C2, const float* w, const float* w2, void* packed, cudaStream_t st);
+cudaError_t igemm_block_forward(const Shape& s, int C2, const float* x, const void* packed, float* y2, Status* status, int sm_count,
+                                cudaStream_t st);
 size_t igemm_scratch_bytes(const Shape& s);   // device scratch the forward needs (padded copy of x), 0 for most shapes
 cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
                           cudaStream_t st, float* scratch);

@@ -52,6 +52,8 @@ constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issu
 constexpr int kThreads = 32 * (kMmaWarp3 + 2);
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
+// Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
+constexpr int kLayoutSMs = 148;
 constexpr uint32_t kPrefetchUses = 1;   // stages whose input is prefetched into L2 before the dependency wait
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr int kMaxDynSmem = 226 * 1024;   // 227 KB per CTA minus the static control block (under 1 KB)
@@ -64,6 +66,9 @@ struct __align__(8) SharedCtl {
     unsigned long long xchg_bar[kMaxAcc];
     unsigned long long b_full[2];   // resident weights of a (group, filter tile) have landed
     unsigned long long b_free[2];   // every MMA that read that weight buffer has completed
+    // fused grouped + pointwise block: the grouped result of a tile goes through shared memory (a2, one buffer per
+    // epilogue group) into a second MMA that accumulates the pointwise output of the pixel tile over all groups (d2)
+    unsigned long long a2_full[2], a2_free[2], d2_full, d2_free, w2_full;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -192,7 +197,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
 // fastest (a CTA keeps its weights across consecutive tiles); with streamed weights the filter tile runs fastest, so
 // the NT tiles that read the same input block run at the same time and the re-reads hit L2 instead of HBM.
 __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, uint32_t& gn, uint32_t& mt) {
-    if (c.nt_fast) {
+    if (c.fuse) {                     // fused block: group fastest, a CTA takes all groups of a pixel tile in turn
+        c.div_ngn.divmod(tile, mt, gn);
+    } else if (c.nt_fast) {
         uint32_t gm, nt, g;
         c.div_nt.divmod(tile, gm, nt);
         c.div_mt.divmod(gm, g, mt);
@@ -209,26 +216,26 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4, tapb;
+        nt_fast, wseg, nseg, SR, fast4, tapb, fuse;
 };
 constexpr int kFamilies = 11;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0}     // row boxes of one segment, narrow groups
-         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1}     // 16x16 / 8x8 planes, narrow groups, tap blocks
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0}     // row boxes of one segment, narrow groups
+         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -281,6 +288,13 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
         } else if (t == 18) {
             ctl.abort_flag = 0;
+        } else if (t >= 20 && t < 22) {
+            mbar_init(smem_u32(&ctl.a2_full[t - 20]), kEpiWarps);
+            mbar_init(smem_u32(&ctl.a2_free[t - 20]), 1);
+        } else if (t == 22) {
+            mbar_init(smem_u32(&ctl.d2_full), 1);
+            mbar_init(smem_u32(&ctl.d2_free), kEpiWarps);
+            mbar_init(smem_u32(&ctl.w2_full), 1);
         }
         if (t >= 0 && t < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -299,6 +313,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     // the CTAs split into one set per pair, each set striding over that pair's pixel tiles: no CTA ever switches
     // weights, and the CTAs of a set still read neighbouring pixels at the same time.
     int tile_first = (int)blockIdx.x, tile_end = c.num_tiles, tile_step = (int)gridDim.x;
+    if (c.fuse) tile_first = (int)blockIdx.x * c.n_gn;    // tile = pixel tile * n_gn + group; see tile_next
+    // next tile of this CTA: every gridDim.x-th tile, or (fused block) the next group of the pixel tile and, after
+    // its last group, the first group of the pixel tile gridDim.x further on
+    auto tile_next = [&](int tile) -> int {
+        if (!c.fuse) return tile + tile_step;
+        uint32_t mt, gn;
+        c.div_ngn.divmod((uint32_t)tile, mt, gn);
+        return (int)gn + 1 == c.n_gn ? tile + 1 + ((int)gridDim.x - 1) * c.n_gn : tile + 1;
+    };
     if (c.cps > 0) {
         const int set = (int)blockIdx.x / c.cps;
         tile_first = set * c.MT + ((int)blockIdx.x - set * c.cps);
@@ -348,6 +371,16 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             cur_gn = (int)gn;
             switches = 1;
         }
+        if (c.fuse) {
+            // the pointwise weights of every group stay resident (they come from the packing kernel too)
+            const uint32_t bar = smem_u32(&ctl.w2_full);
+            const uint32_t w2_blk = (uint32_t)c.Kt * (uint32_t)c.C2 * 4u;
+            if (lane == 0) mbar_arrive_expect_tx(bar, w2_blk * (uint32_t)c.n_gn);
+            __syncwarp();
+            for (int blk = lane; blk < c.n_gn; blk += 32)
+                bulk_load_1d(smem_base + c.w2_off + (uint32_t)blk * w2_blk,
+                             reinterpret_cast<const uint8_t*>(packed) + c.w2_goff + (size_t)blk * w2_blk, w2_blk, bar);
+        }
         // Two passes over the tiles.  Pass 0 runs before the dependency wait and only asks L2 to fetch the input box of
         // the first stage: a cache hint, nothing is consumed, and L2 is the point of coherence, so it stays correct if
         // the previous kernel is still writing those lines (then they are in L2 already).  The CTA usually sits in the
@@ -362,7 +395,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             stage = 0;
             ph = 0;
         }
-        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile += tile_step) {
+        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile = tile_next(tile)) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
             uint32_t gq = gn, ntq = 0;
@@ -477,6 +510,40 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     if (mbar_try_wait(bar, par)) break;
             }
         }
+    } else if (c.fuse && warp == kMmaWarp3) {
+        // ---------------------------------------------------------------- pointwise MMA issuer (fused block)
+        // D2[128 pixels, C2] += A2[128 pixels, Kt] * W2[group][Kt, C2] for every group of the pixel tile in turn; A2 is the
+        // grouped result the epilogue warps wrote to shared memory in the MN-major operand layout.
+        if (lane == 0) {
+            bool ok = mbar_wait(smem_u32(&ctl.w2_full), 0, abort_flag, status, 900);
+            const uint32_t idesc2 = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((uint32_t)(c.C2 >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t a2_blk = (uint32_t)c.Kt * 128u;                      // one 32-pixel block of A2
+            const uint64_t a2_desc0 = make_desc(0, a2_blk, 512u, 1u);
+            const uint32_t b2_lbo = (uint32_t)(c.C2 >> 3) * 128u;
+            const uint64_t b2_desc0 = make_desc(0, b2_lbo, 128u, 0u);
+            const uint32_t a2_hi = (uint32_t)(a2_desc0 >> 32), a2_lo0 = (uint32_t)a2_desc0;
+            const uint32_t b2_hi = (uint32_t)(b2_desc0 >> 32), b2_lo0 = (uint32_t)b2_desc0;
+            const uint32_t w2_blk = (uint32_t)c.Kt * (uint32_t)c.C2 * 4u;
+            const uint32_t d2 = tmem_base + (uint32_t)c.d2_col;
+            uint32_t uses[2] = {0u, 0u}, ptiles = 0, e = 0;
+            for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile), e ^= 1u) {
+                uint32_t gn, mt;
+                tile_coords(c, (uint32_t)tile, gn, mt);
+                if (!mbar_wait(smem_u32(&ctl.a2_full[e]), uses[e] & 1u, abort_flag, status, 910 + (int)e)) break;
+                if (gn == 0 && ptiles > 0 && !mbar_wait(smem_u32(&ctl.d2_free), (ptiles - 1) & 1u, abort_flag, status, 920)) break;
+                tc_fence_after();
+                uint32_t al = a2_lo0 + ((smem_base + c.a2_off + e * 4u * a2_blk) >> 4);
+                uint32_t bl = b2_lo0 + ((smem_base + c.w2_off + gn * w2_blk) >> 4);
+                for (int k8 = 0; k8 < c.Kt / 8; ++k8, al += 64u, bl += (2u * b2_lbo) >> 4)
+                    umma_tf32_split(d2, al, a2_hi, bl, b2_hi, idesc2, (gn != 0 || k8 != 0) ? 1u : 0u);
+                umma_commit(smem_u32(&ctl.a2_free[e]));
+                ++uses[e];
+                if ((int)gn + 1 == c.n_gn) {
+                    umma_commit(smem_u32(&ctl.d2_full));
+                    ++ptiles;
+                }
+            }
+        }
     } else if (warp == 1 || warp == kMmaWarp2 || warp >= kMmaWarp3) {
         // ---------------------------------------------------------------- MMA issuers
         // Two warps issue alternate tiles (each owns one TMEM buffer), so the barrier waits and descriptor
@@ -510,7 +577,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             uint32_t bres_addr = 0;
             bool ok = true;
             for (int tile = tile_first; tile < tile_end && ok;
-                 tile += tile_step, ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u),
+                 tile = tile_next(tile), ++tcount, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u),
                      turn = (turn + 1 == (uint32_t)c.issuers ? 0u : turn + 1)) {
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
@@ -576,10 +643,18 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         const int kbeg = half == 0 ? 0 : kh;
         const int kend = half == 0 ? kh : Kt;
         uint32_t buf = 0, bph = 0, tpar = 0;
+        uint32_t a2_uses = 0, ptiles = 0, d2_seen = 0;   // fused block: uses of this group's A2 buffer, pixel tiles finished,
+                                                         // phases of d2_full this group has observed
         for (int tile = tile_first; tile < tile_end;
-             tile += tile_step, tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
-            if (c.egroups == 2 && tpar != egroup) continue;   // the other group's tile
+             tile = tile_next(tile), tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
             uint32_t gn, mt;
+            if (c.egroups == 2 && tpar != egroup) {           // the other group's tile
+                if (c.fuse) {
+                    tile_coords(c, (uint32_t)tile, gn, mt);
+                    if ((int)gn + 1 == c.n_gn) ++ptiles;
+                }
+                continue;
+            }
             tile_coords(c, (uint32_t)tile, gn, mt);
             uint32_t n, i;
             int f;
@@ -629,6 +704,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint32_t t0 = tmem_base + buf * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
             // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
             float* yk = y + ((size_t)n * s.C_out + (size_t)gn * Kt + (size_t)kbeg) * OHW + fo;
+            // fused block: this lane's slot in the A2 operand (32-pixel block wq, 128-byte row per channel, 32-byte
+            // chunks swizzled by the channel index), once the pointwise MMAs of the buffer's previous use are done
+            uint8_t* a2p = smem + c.a2_off + (size_t)egroup * 4u * (size_t)Kt * 128u + (size_t)wq * (size_t)Kt * 128u + (size_t)(lane & 7) * 4u;
+            if (c.fuse && a2_uses > 0 && !mbar_wait_warp(smem_u32(&ctl.a2_free[egroup]), (a2_uses - 1) & 1u, abort_flag, status, 930)) break;
             if (c.need_xchg) {
                 // Rows may straddle a warp boundary: publish this warp's edge lanes (lane 31's left-tap
                 // and lane 0's right-tap accumulators) so the neighbouring quarter can add them, then wait
@@ -665,13 +744,51 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     if (add_dn) v += dn;
                     if (edge_up) v += xchg[buf][wq - 1][0][k0 + j];
                     if (edge_dn) v += xchg[buf][wq + 1][1][k0 + j];
-                    if (valid) *yk = v;
-                    yk += OHW;
+                    if (c.fuse) {
+                        const int k = k0 + j;
+                        *reinterpret_cast<float*>(a2p + (size_t)k * 128u + (size_t)((((uint32_t)lane >> 3) ^ ((uint32_t)k & 3u)) << 5)) = v;
+                    } else {
+                        if (valid) *yk = v;
+                        yk += OHW;
+                    }
                 }
             }
+            if (c.fuse) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads A2 through the async proxy
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+            if (c.fuse) {
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.a2_full[egroup]));
+                ++a2_uses;
+                if ((int)gn + 1 == c.n_gn) {
+                    // last group of the pixel tile: its pointwise result is complete once the MMAs just requested are done
+                    // (a parity wait is only meaningful one phase at a time: first observe, in order, the phases of the
+                    // pixel tiles the other group finished)
+                    bool ok2 = true;
+                    for (; d2_seen <= ptiles && ok2; ++d2_seen)
+                        ok2 = mbar_wait_warp(smem_u32(&ctl.d2_full), d2_seen & 1u, abort_flag, status, 940);
+                    if (!ok2) break;
+                    tc_fence_after();
+                    const uint32_t d2 = tmem_base + (uint32_t)c.d2_col + ((uint32_t)(wq * 32) << 16);
+                    const int c2h = ((c.C2 / 2) + 7) & ~7;
+                    const int c2beg = half == 0 ? 0 : c2h, c2end = half == 0 ? c2h : c.C2;
+                    float* y2 = y + ((size_t)n * c.C2 + (size_t)c2beg) * OHW + fo;
+                    for (int k0 = c2beg; k0 < c2end; k0 += 8) {
+                        float d[8];
+                        tmem_ld8(d2 + (uint32_t)k0, d);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (valid) *y2 = d[j];
+                            y2 += OHW;
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl.d2_free));
+                    ++ptiles;
+                }
+            }
         }
     }
 
@@ -843,8 +960,9 @@ size_t igemm_scratch_bytes(const Shape& s) {
     return ge.padded ? sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp : 0;
 }
 
-IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
+static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
     IgemmCfg c;
+    const bool fuse = C2 > 0;          // fused grouped + pointwise block: heavy shape, streamed or resident grouped weights
     const IgemmGeom ge = igemm_geom(s_true);
     Shape s = s_true;          // the plane the kernel computes on
     s.H = ge.Hp;
@@ -944,7 +1062,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     // segments, each loaded with its own row shift -- so a tile costs one barrier round trip instead of three.  Only
     // where a tile straddles images anyway (8x8): 16x16 planes keep their one-box-per-tap copies, which are faster.
     c.tapb = 0;
-    if (c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
+    if (!fuse && c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
         3u * (uint32_t)c.Cg * (uint32_t)c.Np * 4u <= 40u * 1024u) {
         c.tapb = 1;
         c.nr = 3;
@@ -973,12 +1091,19 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
         const uint32_t a_only = (a_bytes + 1023u) & ~1023u;
         if (c.b_res == 1 && c.bres_stride + 2u * a_only + xchg_bytes + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
         // loading a large filter bank up front only pays when a CTA reuses it over several pixel tiles
-        if (c.b_res == 1 && b_tile > 40u * 1024u && c.MT < 4 * sm_count) c.b_res = 0;
+        if (!fuse && c.b_res == 1 && b_tile > 40u * 1024u && c.MT < 4 * sm_count) c.b_res = 0;
     }
+    if (fuse && c.b_res == 1 && c.groups * c.NT > 1) c.b_res = 0;   // the group changes every tile: stream, or two buffers
     c.egroups = 2;
     c.threads = kThreads;
     c.tmem_cols = kTmemCols;
     uint32_t budget_total = 200u * 1024u;
+    const uint32_t w2_bytes = fuse ? (uint32_t)c.groups * (uint32_t)c.Kt * (uint32_t)C2 * 4u : 0u;   // resident pointwise weights
+    const uint32_t a2_bytes = fuse ? 2u * 4u * (uint32_t)c.Kt * 128u : 0u;                             // two A2 operand buffers
+    if (fuse) {
+        budget_total = (uint32_t)kMaxDynSmem - 2048u - w2_bytes - a2_bytes;
+        c.nacc = 2;
+    }
     // Light configuration, two CTAs per SM: one epilogue group, two accumulators in 256 TMEM columns, one resident
     // weight buffer and half the shared memory.  The two CTAs hide each other's start-up, barrier and drain
     // latencies, and a CTA of the next kernel in the stream can start while one of this kernel's is still at work.
@@ -986,7 +1111,7 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
         const uint32_t light_total = 110u * 1024u;
         const uint32_t st_bytes = (a_bytes + 1023u) & ~1023u;
         const int kst = (3 / c.nr) * c.chunks;
-        const bool fits = 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
+        const bool fits = !fuse && 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
                           c.bres_stride + (uint32_t)(c.tapb ? 1 : (kst == 1 ? 2 : kst + 1)) * st_bytes + xchg_bytes + 1024u <= light_total;
         if (fits) {
             c.b_res = 1;
@@ -1014,15 +1139,81 @@ IgemmCfg igemm_config(const Shape& s_true, int sm_count) {
     // into one set per pair and no CTA ever switches (two buffers hide the switch; there the plain order keeps all
     // SMs busy and balanced).
     c.cps = 0;
+    c.fuse = fuse ? 1 : 0;
+    c.C2 = C2;
+    c.n_gn = c.groups * c.NT;
+    c.div_ngn = make_fastdiv((uint32_t)c.n_gn);
+    c.d2_col = c.nacc * c.Np;
+    c.w2_off = (uint32_t)c.smem_bytes - 1024u;             // behind the stages (and the exchange area)
+    c.a2_off = c.w2_off + ((w2_bytes + 1023u) & ~1023u);
+    c.w2_goff = kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    if (fuse) {
+        c.smem_bytes = (size_t)c.a2_off + a2_bytes + 1024;
+        c.issuers = 2;
+        c.grid = c.MT < sm_count ? c.MT : sm_count;        // a CTA takes whole pixel tiles (all groups of each)
+    }
     {
         const int n_gn = c.groups * c.NT;
-        if (c.b_res == 1 && n_gn > 1 && c.grid >= n_gn) {
+        if (!fuse && c.b_res == 1 && n_gn > 1 && c.grid >= n_gn) {
             c.cps = c.grid / n_gn;                   // CTAs per (group, filter tile)
             if (c.cps > c.MT) c.cps = c.MT;
             c.grid = c.cps * n_gn;
         }
     }
     return c;
+}
+
+IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, sm_count, 0); }
+
+// ---- fused block: grouped 3x3 followed by a pointwise (1x1, groups = 1) convolution C_out -> C2 ------------------------
+bool igemm_block_supported(const Shape& s, int C2) {
+    if (!igemm_supported(s) || s.stride != 1 || C2 < 16 || C2 % 16 != 0) return false;
+    const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
+    if (c.NT != 1 || c.need_xchg || c.padded || c.egroups != 2 || c.nacc != 2) return false;
+    if (c.d2_col + C2 > kTmemCols) return false;
+    if ((uint32_t)c.groups * (uint32_t)c.Kt * (uint32_t)C2 * 4u >= (1u << 20)) return false;   // one barrier phase takes the whole of W2
+    return c.stages >= 2 && c.smem_bytes <= (size_t)kMaxDynSmem;
+}
+
+size_t igemm_block_packed_bytes(const Shape& s, int C2) {
+    const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
+    return c.w2_goff + sizeof(float) * (size_t)c.groups * c.Kt * C2;
+}
+
+namespace {
+// Pointwise weights w2[C2][C_out] -> one K-major operand image per merged group: [k/8][k%8/4][n/8][n%8][4 channels],
+// k = channel of the group's Kt grouped outputs, n = pointwise output channel; values rounded to TF32.
+__global__ void block_pack_w2_kernel(int groups, int Kt, int C2, int C_mid, const float* __restrict__ w2, uint32_t* __restrict__ dst) {
+    const size_t total = (size_t)groups * Kt * C2;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        size_t t = i;
+        const int e = (int)(t % 4); t /= 4;
+        const int n8 = (int)(t % 8); t /= 8;
+        const int nb = (int)(t % (C2 / 8)); t /= (C2 / 8);
+        const int k2 = (int)(t % 2); t /= 2;
+        const int k8 = (int)(t % (Kt / 8));
+        const int g = (int)(t / (Kt / 8));
+        const int k = k8 * 8 + k2 * 4 + e, n = nb * 8 + n8;
+        const float v = w2[(size_t)n * C_mid + (size_t)g * Kt + k];
+        uint32_t u;
+        asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(v));
+        dst[i] = u;
+    }
+}
+}  // namespace
+
+static uint32_t block_tag(const Shape& s, int C2) { return pack_tag(s, GCONV_VARIANT_IGEMM_TF32) ^ (0xB10C0000u + (uint32_t)C2); }
+
+cudaError_t igemm_block_pack(const Shape& s, int C2, const float* w, const float* w2, void* packed, cudaStream_t st) {
+    const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
+    const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
+    igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), block_tag(s, C2));
+    const size_t t2 = (size_t)c.groups * c.Kt * C2;
+    blocks = (int)((t2 + 255) / 256 < 2368 ? (t2 + 255) / 256 : 2368);
+    block_pack_w2_kernel<<<blocks, 256, 0, st>>>(c.groups, c.Kt, C2, s.C_out, w2,
+                                                 reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(packed) + c.w2_goff));
+    return cudaGetLastError();
 }
 
 size_t igemm_packed_bytes(const Shape& s) {
@@ -1038,9 +1229,22 @@ cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_
     return cudaGetLastError();
 }
 
+static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, const void* packed, float* y, Status* status,
+                                int sm_count, cudaStream_t st, float* scratch);
+
 cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* packed, float* y, Status* status, int sm_count,
                           cudaStream_t st, float* scratch) {
-    const IgemmCfg c = igemm_config(s_true, sm_count);
+    return igemm_launch(s_true, 0, x_in, packed, y, status, sm_count, st, scratch);
+}
+
+cudaError_t igemm_block_forward(const Shape& s, int C2, const float* x, const void* packed, float* y2, Status* status, int sm_count,
+                                cudaStream_t st) {
+    return igemm_launch(s, C2, x, packed, y2, status, sm_count, st, nullptr);
+}
+
+static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, const void* packed, float* y, Status* status,
+                                int sm_count, cudaStream_t st, float* scratch) {
+    const IgemmCfg c = igemm_config_c2(s_true, sm_count, C2);
     Shape s = s_true;
     const float* x = x_in;
     if (c.padded) {
@@ -1142,7 +1346,7 @@ cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* pa
     lc.attrs = attr;
     lc.numAttrs = 1;
     return cudaLaunchKernelEx(&lc, kernels[fam], xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
-                              pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32));
+                              C2 > 0 ? block_tag(s_true, C2) : pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32));
 }
 
 

@@ -46,6 +46,10 @@ _SIGNATURES = {
     "gconv_forward": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "gconv_forward_host": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "gconv_forward_host_static": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
+    "gconv_block_supported": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "gconv_block_packed_bytes": (ctypes.c_size_t, [_vp, ctypes.c_int]),
+    "gconv_block_pack_weights": (ctypes.c_int, [_vp, ctypes.c_int, _vp, _vp, _vp, _vp]),
+    "gconv_block_forward": (ctypes.c_int, [_vp, ctypes.c_int, _vp, _vp, _vp, _vp]),
     "gconv_forward_launches": (ctypes.c_int, [_vp]),
     "gconv_last_status": (ctypes.c_int, [_vp, _vp]),
     "gconv_last_cuda_error": (ctypes.c_int, [_vp]),
@@ -164,6 +168,26 @@ def gconv_forward_host_static(desc, x_host, w_packed, y_host, stream=None) -> No
     blocks until y_host is complete and raises on any status other than GCONV_OK."""
     _check(load().gconv_forward_host_static(desc, _ptr(x_host), _ptr(w_packed), _ptr(y_host), _stream(stream)),
            "gconv_forward_host_static")
+
+
+def gconv_block_supported(desc, C2: int) -> bool:
+    return bool(load().gconv_block_supported(desc, int(C2)))
+
+
+def gconv_block_packed_bytes(desc, C2: int) -> int:
+    return int(load().gconv_block_packed_bytes(desc, int(C2)))
+
+
+def gconv_block_pack_weights(desc, C2: int, w_ochw, w2, w_packed, stream=None) -> None:
+    """Packs the grouped 3x3 weights and the pointwise weights [C2, C_out] of the fused block (asynchronous)."""
+    _check(load().gconv_block_pack_weights(desc, int(C2), _ptr(w_ochw), _ptr(w2), _ptr(w_packed), _stream(stream)),
+           "gconv_block_pack_weights")
+
+
+def gconv_block_forward(desc, C2: int, x_nchw, w_packed, y2_nchw, stream=None) -> None:
+    """Grouped 3x3 convolution followed by the pointwise convolution, one kernel (asynchronous)."""
+    _check(load().gconv_block_forward(desc, int(C2), _ptr(x_nchw), _ptr(w_packed), _ptr(y2_nchw), _stream(stream)),
+           "gconv_block_forward")
 
 
 def gconv_forward_launches(desc) -> int:

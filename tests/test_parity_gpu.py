@@ -242,6 +242,60 @@ def test_dependent_chain_back_to_back(shape):
             gconv.gconv_desc_destroy(d)
 
 
+BLOCK_SHAPES = [
+    # N, C_in of the grouped 3x3, H, W, groups, C2 (pointwise outputs) [, C_out of the grouped 3x3 if not C_in]
+    (2, 32, 32, 32, 4, 32), (40, 32, 32, 32, 4, 32), (130, 32, 32, 32, 16, 48), (3, 64, 16, 16, 2, 64), (96, 64, 16, 16, 8, 128),
+    (64, 128, 8, 8, 8, 128), (9, 64, 56, 56, 16, 64), (20, 128, 28, 28, 32, 64), (33, 96, 20, 24, 3, 80), (7, 64, 30, 60, 8, 16),
+    (5, 32, 12, 56, 1, 32, 64), (1, 32, 8, 8, 32, 256), (12, 64, 16, 16, 2, 96, 128),
+]
+
+
+@pytest.mark.parametrize("cfg", BLOCK_SHAPES)
+def test_fused_grouped_pointwise_block(cfg):
+    """The paper's G(g) block in one kernel: grouped 3x3 then pointwise.  Compared with the oracle's grouped convolution
+    (its fp64 result rounded to fp32, as the kernel keeps the intermediate in fp32) followed by its 1x1 convolution."""
+    N, Cin, H, W, groups, C2 = cfg[:6]
+    C = cfg[6] if len(cfg) > 6 else Cin                    # channels between the two convolutions
+    L = Layer("block", N, Cin, H, W, C, groups=groups)
+    dev = torch.device("cuda:0")
+    x, w = synth.make_layer_tensors(N, Cin, H, W, C, 3, 3, groups, synth.layer_seed(41, N, C, groups))
+    _, w2 = synth.make_layer_tensors(1, C, 1, 1, C2, 1, 1, 1, synth.layer_seed(42, C, C2))
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_block_supported(d, C2)
+        guard, sentinel = 64, float(np.float32(-1.2345678e30))
+        pb = gconv.gconv_block_packed_bytes(d, C2)
+        wp_full = torch.full((pb // 4 + 2 * guard,), sentinel, dtype=torch.float32, device=dev)
+        y_full = torch.full((N * C2 * H * W + 2 * guard,), sentinel, dtype=torch.float32, device=dev)
+        wp, y2 = wp_full[guard:guard + pb // 4], y_full[guard:guard + N * C2 * H * W]
+        gconv.gconv_block_pack_weights(d, C2, torch.from_numpy(w).to(dev), torch.from_numpy(w2.reshape(C2, C)).to(dev), wp)
+        xd = torch.from_numpy(x).to(dev)
+        gconv.gconv_block_forward(d, C2, xd, wp, y2)
+        gconv.gconv_block_forward(d, C2, xd, wp, y2)          # back to back: the second starts before the first ends
+        assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+        for band in (wp_full[:guard], wp_full[-guard:], y_full[:guard], y_full[-guard:]):
+            assert bool((band == sentinel).all()), "guard band overwritten"
+        got = y2.cpu().numpy().reshape(N, C2, H, W)
+        y1 = oracle.gconv_ref(x, w, 1, 1, 1, groups, threads=8)
+        ref = oracle.gconv_ref(y1.astype(np.float32), w2, 1, 0, 1, 1, threads=8)
+        assert np.all(np.isfinite(got))
+        assert rel_err(got, ref) <= 5e-3
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def test_fused_block_rejects_what_it_cannot_run():
+    for cfg, C2 in (((1, 32, 32, 32, 32, 3, 3, 2, 1, 1, 4), 32), ((1, 32, 14, 14, 32, 3, 3, 1, 1, 1, 4), 32),
+                    ((1, 32, 32, 32, 32, 3, 3, 1, 1, 1, 4), 24), ((1, 256, 28, 28, 256, 3, 3, 1, 1, 1, 32), 256),
+                    ((1, 32, 32, 32, 32, 5, 5, 1, 2, 1, 32), 32)):
+        d = gconv.gconv_desc_create(*cfg)
+        try:
+            assert not gconv.gconv_block_supported(d, C2)
+            assert gconv.gconv_block_packed_bytes(d, C2) == 0
+        finally:
+            gconv.gconv_desc_destroy(d)
+
+
 def test_pack_mismatch_is_reported_not_fatal():
     (L,) = config0()
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 5)
