@@ -288,10 +288,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
         } else if (t == 18) {
             ctl.abort_flag = 0;
-        } else if (t >= 20 && t < 22) {
+        } else if (c.fuse && t >= 20 && t < 22) {
             mbar_init(smem_u32(&ctl.a2_full[t - 20]), kEpiWarps);
             mbar_init(smem_u32(&ctl.a2_free[t - 20]), 1);
-        } else if (t == 22) {
+        } else if (c.fuse && t == 22) {
             mbar_init(smem_u32(&ctl.d2_full), 1);
             mbar_init(smem_u32(&ctl.d2_free), kEpiWarps);
             mbar_init(smem_u32(&ctl.w2_full), 1);
