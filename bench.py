@@ -232,6 +232,65 @@ def time_layer(torch, gconv, L, stream, reps=160, min_cycle_bytes=2 * L2_BYTES +
         gconv.gconv_desc_destroy(d)
 
 
+def time_block(torch, gconv, L, C2, stream, reps=20, min_cycle_bytes=2 * L2_BYTES + (64 << 20)):
+    """Average device time of one gconv_block_forward launch (grouped 3x3 of layer L, then pointwise C_out -> C2)
+    with cold L2, timed like time_layer; None when the fused kernel does not take the shape."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    y2_elems = L.N * C2 * L.H_out * L.W_out
+    per = 4 * (L.x_elems + y2_elems)
+    nbuf = max(2, -(-min_cycle_bytes // per))
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        if not gconv.gconv_block_supported(d, C2):
+            return None
+        x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.groups, 99, L.x_dist)
+        _, w2 = synth.make_layer_tensors(1, L.C_out, 1, 1, C2, 1, 1, 1, 98)
+        reps_x = -(-L.N // x0.shape[0])
+        xs = [torch.from_numpy(x0).to(dev).repeat(reps_x, 1, 1, 1)[:L.N].contiguous() for _ in range(nbuf)]
+        ys = [torch.empty(y2_elems, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+        wp = torch.empty(gconv.gconv_block_packed_bytes(d, C2) // 4, dtype=torch.float32, device=dev)
+        with torch.cuda.stream(stream):
+            gconv.gconv_block_pack_weights(d, C2, torch.from_numpy(w0).to(dev), torch.from_numpy(w2.reshape(C2, L.C_out)).to(dev), wp, stream)
+            for i in range(min(nbuf, 5) + 3):
+                gconv.gconv_block_forward(d, C2, xs[i % nbuf], wp, ys[i % nbuf], stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            graph = torch.cuda.CUDAGraph()
+            stream.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(reps):
+                    gconv.gconv_block_forward(d, C2, xs[i % nbuf], wp, ys[i % nbuf], stream)
+            graph.replay()
+            stream.synchronize()
+            times = []
+            for _ in range(5):
+                e0.record(stream)
+                graph.replay()
+                e1.record(stream)
+                stream.synchronize()
+                times.append(e0.elapsed_time(e1) / reps)
+        st = gconv.gconv_last_status(d, stream)
+        assert st == 0, gconv.status_string(st)
+        return statistics.median(times)
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def block_row(L, C2, ms_block, ms_grouped, peaks):
+    """Fused grouped + pointwise block: its time against the HBM floor of the block (x in, y2 out) and against the
+    unfused pair's floor (the grouped layer as measured alone, plus reading y1 and writing y2 at the HBM peak)."""
+    hbm = peaks["hbm_gbs"] * 1e9
+    pix = L.N * L.H_out * L.W_out
+    bytes_block = 4 * (L.x_elems + pix * C2)
+    flops = L.flops + 2 * pix * L.C_out * C2
+    t_tensor = flops / (0.5 * peaks["bf16_tflops"] * 1e12)
+    t_roof = max(bytes_block / hbm, t_tensor)
+    unfused_floor_ms = ms_grouped + 4e3 * pix * (L.C_out + C2) / hbm
+    return {"layer": L.name, "groups": L.groups, "N": L.N, "C2": C2, "ms": ms_block, "grouped_only_ms": ms_grouped,
+            "unfused_floor_ms": unfused_floor_ms, "gflops": flops / (ms_block * 1e-3) / 1e9,
+            "gbs": bytes_block / (ms_block * 1e-3) / 1e9, "roofline_ms": t_roof * 1e3,
+            "bound": "hbm" if bytes_block / hbm >= t_tensor else "tensor", "roofline_frac": t_roof / (ms_block * 1e-3)}
+
+
 def chained_stack_ms(torch, gconv, groups, stream, reps=50):
     """Batch-1 inference over the 18-layer stack as a real chain (each layer reads the previous layer's output),
     replayed as one CUDA graph: ms per pass.  This is the shape of the paper's whole-network timings (N = 1),
@@ -459,6 +518,13 @@ def run_ours(args):
                 ms, v = time_layer(torch, gconv, L, stream, reps=20)
                 sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
             extra["sweep_layers"] = sweep_rows
+            block_rows = []
+            for L, C2 in wl.fused_blocks():
+                msb = time_block(torch, gconv, L, C2, stream)
+                if msb is not None:
+                    msg, _ = time_layer(torch, gconv, L, stream, reps=20)
+                    block_rows.append(block_row(L, C2, msb, msg, peaks))
+            extra["fused_blocks"] = block_rows
             extra["stack_n1_chained_ms_by_groups"] = {str(g): chained_stack_ms(torch, gconv, g, stream) for g in wl.WRN_GROUPS}
 
     # ---- CPU baseline (rank 0, N=1 only) -----------------------------------------------------------

@@ -68,7 +68,7 @@ struct __align__(8) SharedCtl {
     unsigned long long b_free[2];   // every MMA that read that weight buffer has completed
     // fused grouped + pointwise block: the grouped result of a tile goes through shared memory (a2, one buffer per
     // epilogue group) into a second MMA that accumulates the pointwise output of the pixel tile over all groups (d2)
-    unsigned long long a2_full[2], a2_free[2], d2_full, d2_free, w2_full;
+    unsigned long long a2_full[2], a2_free[2], d2_full[2], d2_free[2], w2_full;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -218,7 +218,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse;
 };
-constexpr int kFamilies = 11;
+constexpr int kFamilies = 13;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -231,6 +231,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
          : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0}     // row boxes of one segment, narrow groups
          : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1}     // fused block, 32-wide planes with halo stages
+         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1}     // fused block, 16x16 / 8x8 planes, two resident banks
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -292,9 +294,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             mbar_init(smem_u32(&ctl.a2_full[t - 20]), kEpiWarps);
             mbar_init(smem_u32(&ctl.a2_free[t - 20]), 1);
         } else if (c.fuse && t == 22) {
-            mbar_init(smem_u32(&ctl.d2_full), 1);
-            mbar_init(smem_u32(&ctl.d2_free), kEpiWarps);
             mbar_init(smem_u32(&ctl.w2_full), 1);
+        } else if (c.fuse && t >= 24 && t < 26) {
+            mbar_init(smem_u32(&ctl.d2_full[t - 24]), 1);
+            mbar_init(smem_u32(&ctl.d2_free[t - 24]), kEpiWarps);
         }
         if (t >= 0 && t < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -524,13 +527,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint32_t a2_hi = (uint32_t)(a2_desc0 >> 32), a2_lo0 = (uint32_t)a2_desc0;
             const uint32_t b2_hi = (uint32_t)(b2_desc0 >> 32), b2_lo0 = (uint32_t)b2_desc0;
             const uint32_t w2_blk = (uint32_t)c.Kt * (uint32_t)c.C2 * 4u;
-            const uint32_t d2 = tmem_base + (uint32_t)c.d2_col;
             uint32_t uses[2] = {0u, 0u}, ptiles = 0, e = 0;
             for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile), e ^= 1u) {
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
                 if (!mbar_wait(smem_u32(&ctl.a2_full[e]), uses[e] & 1u, abort_flag, status, 910 + (int)e)) break;
-                if (gn == 0 && ptiles > 0 && !mbar_wait(smem_u32(&ctl.d2_free), (ptiles - 1) & 1u, abort_flag, status, 920)) break;
+                // the pixel tile's accumulator: two of them take alternate pixel tiles when TMEM has the room
+                const uint32_t db = c.d2_bufs == 2 ? (ptiles & 1u) : 0u, du = c.d2_bufs == 2 ? (ptiles >> 1) : ptiles;
+                const uint32_t d2 = tmem_base + (uint32_t)c.d2_col + db * (uint32_t)c.C2;
+                if (gn == 0 && du > 0 && !mbar_wait(smem_u32(&ctl.d2_free[db]), (du - 1) & 1u, abort_flag, status, 920)) break;
                 tc_fence_after();
                 uint32_t al = a2_lo0 + ((smem_base + c.a2_off + e * 4u * a2_blk) >> 4);
                 uint32_t bl = b2_lo0 + ((smem_base + c.w2_off + gn * w2_blk) >> 4);
@@ -539,7 +544,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 umma_commit(smem_u32(&ctl.a2_free[e]));
                 ++uses[e];
                 if ((int)gn + 1 == c.n_gn) {
-                    umma_commit(smem_u32(&ctl.d2_full));
+                    umma_commit(smem_u32(&ctl.d2_full[db]));
                     ++ptiles;
                 }
             }
@@ -645,6 +650,33 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         uint32_t buf = 0, bph = 0, tpar = 0;
         uint32_t a2_uses = 0, ptiles = 0, d2_seen = 0;   // fused block: uses of this group's A2 buffer, pixel tiles finished,
                                                          // phases of d2_full this group has observed
+        // Fused block, second epilogue: the pointwise result of pixel tile p (accumulator p % d2_bufs) goes to y2.  With two
+        // accumulators it is deferred until the group has handed its next grouped result to the tensor core, so the
+        // group never idles through the pointwise MMAs' latency; pend_* remember the deferred tile.
+        bool pend = false, pend_valid = false;
+        uint32_t pend_p = 0;
+        float* pend_y2 = nullptr;
+        const int c2h = ((c.C2 / 2) + 7) & ~7;
+        const int c2beg = half == 0 ? 0 : c2h, c2end = half == 0 ? c2h : c.C2;
+        auto epilogue2 = [&](uint32_t db, uint32_t parity, float* y2, bool v) -> bool {
+            if (!mbar_wait_warp(smem_u32(&ctl.d2_full[db]), parity, abort_flag, status, 940)) return false;
+            tc_fence_after();
+            const uint32_t d2 = tmem_base + (uint32_t)c.d2_col + db * (uint32_t)c.C2 + ((uint32_t)(wq * 32) << 16);
+            for (int k0 = c2beg; k0 < c2end; k0 += 8) {
+                float d[8];
+                tmem_ld8(d2 + (uint32_t)k0, d);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (v) *y2 = d[j];
+                    y2 += OHW;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.d2_free[db]));
+            return true;
+        };
         for (int tile = tile_first; tile < tile_end;
              tile = tile_next(tile), tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
             uint32_t gn, mt;
@@ -760,36 +792,34 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             if (c.fuse) {
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.a2_full[egroup]));
                 ++a2_uses;
-                if ((int)gn + 1 == c.n_gn) {
-                    // last group of the pixel tile: its pointwise result is complete once the MMAs just requested are done
-                    // (a parity wait is only meaningful one phase at a time: first observe, in order, the phases of the
-                    // pixel tiles the other group finished)
-                    bool ok2 = true;
-                    for (; d2_seen <= ptiles && ok2; ++d2_seen)
-                        ok2 = mbar_wait_warp(smem_u32(&ctl.d2_full), d2_seen & 1u, abort_flag, status, 940);
-                    if (!ok2) break;
-                    tc_fence_after();
-                    const uint32_t d2 = tmem_base + (uint32_t)c.d2_col + ((uint32_t)(wq * 32) << 16);
-                    const int c2h = ((c.C2 / 2) + 7) & ~7;
-                    const int c2beg = half == 0 ? 0 : c2h, c2end = half == 0 ? c2h : c.C2;
-                    float* y2 = y + ((size_t)n * c.C2 + (size_t)c2beg) * OHW + fo;
-                    for (int k0 = c2beg; k0 < c2end; k0 += 8) {
-                        float d[8];
-                        tmem_ld8(d2 + (uint32_t)k0, d);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (valid) *y2 = d[j];
-                            y2 += OHW;
-                        }
+                float* y2_tile = y + ((size_t)n * c.C2 + (size_t)c2beg) * OHW + fo;
+                const bool last_gn = (int)gn + 1 == c.n_gn;   // the pixel tile's pointwise result is complete once the MMAs just requested are done
+                if (c.d2_bufs == 2) {
+                    // each accumulator's phases are seen in order by one group: group p % 2 when n_gn is odd, else the second
+                    if (pend) {
+                        if (!epilogue2(pend_p & 1u, (pend_p >> 1) & 1u, pend_y2, pend_valid)) break;
+                        pend = false;
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl.d2_free));
+                    if (last_gn) {
+                        pend = true;
+                        pend_p = ptiles;
+                        pend_y2 = y2_tile;
+                        pend_valid = valid;
+                        ++ptiles;
+                    }
+                } else if (last_gn) {
+                    // one accumulator, both groups wait on the same barrier: a parity wait is only meaningful one phase at
+                    // a time, so first observe, in order, the phases of the pixel tiles the other group finished
+                    bool ok2 = true;
+                    for (; d2_seen < ptiles && ok2; ++d2_seen)
+                        ok2 = mbar_wait_warp(smem_u32(&ctl.d2_full[0]), d2_seen & 1u, abort_flag, status, 941);
+                    if (!ok2 || !epilogue2(0u, d2_seen & 1u, y2_tile, valid)) break;
+                    ++d2_seen;
                     ++ptiles;
                 }
             }
         }
+        if (c.fuse && pend && !*abort_flag) epilogue2(pend_p & 1u, (pend_p >> 1) & 1u, pend_y2, pend_valid);
     }
 
     tc_fence_before();
@@ -1144,6 +1174,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
     c.n_gn = c.groups * c.NT;
     c.div_ngn = make_fastdiv((uint32_t)c.n_gn);
     c.d2_col = c.nacc * c.Np;
+    c.d2_bufs = (fuse && c.d2_col + 2 * C2 <= kTmemCols) ? 2 : 1;
     c.w2_off = (uint32_t)c.smem_bytes - 1024u;             // behind the stages (and the exchange area)
     c.a2_off = c.w2_off + ((w2_bytes + 1023u) & ~1023u);
     c.w2_goff = kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
@@ -1167,7 +1198,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, 
 
 // ---- fused block: grouped 3x3 followed by a pointwise (1x1, groups = 1) convolution C_out -> C2 ------------------------
 bool igemm_block_supported(const Shape& s, int C2) {
-    if (!igemm_supported(s) || s.stride != 1 || C2 < 16 || C2 % 16 != 0) return false;
+    if (!igemm_supported(s) || s.stride != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
     if (c.NT != 1 || c.need_xchg || c.padded || c.egroups != 2 || c.nacc != 2) return false;
     if (c.d2_col + C2 > kTmemCols) return false;
@@ -1323,7 +1354,8 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     static const KernelFn kernels[kFamilies] = {igemm_tf32_kernel<0>, igemm_tf32_kernel<1>, igemm_tf32_kernel<2>,
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
-                                                igemm_tf32_kernel<9>, igemm_tf32_kernel<10>};
+                                                igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
+                                                igemm_tf32_kernel<12>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;

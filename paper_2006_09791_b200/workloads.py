@@ -149,3 +149,17 @@ def depthwise5x5_layers(N: int = 64) -> List[Layer]:
     widths 72...960.  The second depthwise family of the follow-up items."""
     mk = lambda C, HW, s: Layer("dw5_%d@%d%s" % (C, HW, "s2" if s == 2 else ""), N, C, HW, HW, C, 5, 5, s, 2, 1, C)
     return [mk(72, 56, 2), mk(120, 28, 1), mk(240, 28, 2), mk(672, 14, 1), mk(672, 14, 2), mk(960, 7, 1)]
+
+
+def fused_blocks(N: int = 128):
+    """(grouped 3x3 layer, pointwise output channels) pairs of the paper's G(g) block -- a grouped 3x3 followed by a
+    pointwise convolution (Section II) -- at the three stages of the WRN-40-2-shaped stack, plus two ResNeXt-shaped
+    blocks whose pointwise convolution widens the channels."""
+    out = []
+    for g in (2, 4, 8, 16):
+        out.append((Layer("blk32@32", N, 32, 32, 32, 32, groups=g), 32))
+    out.append((Layer("blk64@16", N, 64, 16, 16, 64, groups=4), 64))
+    out.append((Layer("blk128@8", N, 128, 8, 8, 128, groups=8), 128))
+    out.append((Layer("blk128@56", N // 2, 128, 56, 56, 128, groups=32), 256))
+    out.append((Layer("blk64@56", N // 2, 64, 56, 56, 64, groups=16), 256))
+    return out

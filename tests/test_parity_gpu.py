@@ -287,7 +287,7 @@ def test_fused_grouped_pointwise_block(cfg):
 def test_fused_block_rejects_what_it_cannot_run():
     for cfg, C2 in (((1, 32, 32, 32, 32, 3, 3, 2, 1, 1, 4), 32), ((1, 32, 14, 14, 32, 3, 3, 1, 1, 1, 4), 32),
                     ((1, 32, 32, 32, 32, 3, 3, 1, 1, 1, 4), 24), ((1, 256, 28, 28, 256, 3, 3, 1, 1, 1, 32), 256),
-                    ((1, 32, 32, 32, 32, 5, 5, 1, 2, 1, 32), 32)):
+                    ((1, 32, 32, 32, 32, 5, 5, 1, 2, 1, 32), 32), ((1, 32, 8, 8, 32, 3, 3, 1, 1, 1, 32), 272)):
         d = gconv.gconv_desc_create(*cfg)
         try:
             assert not gconv.gconv_block_supported(d, C2)
