@@ -216,28 +216,29 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4, tapb, fuse;
+        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball;
 };
-constexpr int kFamilies = 13;
+constexpr int kFamilies = 14;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0}     // row boxes of one segment, narrow groups
-         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
-         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1}     // fused block, 32-wide planes with halo stages
-         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1}     // fused block, 16x16 / 8x8 planes, two resident banks
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0}     // row boxes of one segment, narrow groups
+         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes with halo stages
+         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
+         : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes, two CTAs per SM
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -373,6 +374,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 bulk_load_1d(bres_base + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
             cur_gn = (int)gn;
             switches = 1;
+            if (c.ball) {
+                // every (group, filter tile) has a resident buffer of its own: fetch the second bank too, nothing ever switches
+                const uint32_t bar1 = smem_u32(&ctl.b_full[1]);
+                if (lane == 0) mbar_arrive_expect_tx(bar1, b_tile_bytes);
+                __syncwarp();
+                for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                    bulk_load_1d(bres_base + c.bres_stride + blk * blk_bytes, wblocks + (size_t)b_tile_bytes + (size_t)blk * blk_bytes, blk_bytes, bar1);
+                switches = 2;
+            }
         }
         if (c.fuse) {
             // the pointwise weights of every group stay resident (they come from the packing kernel too)
@@ -405,7 +415,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             if (c.NT > 1) c.div_nt.divmod(gn, gq, ntq);
             const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
-            const bool switch_b = !pf && c.b_res && (int)gn != cur_gn;
+            const bool switch_b = !pf && c.b_res && !c.ball && (int)gn != cur_gn;
             // Whole-tile copies: a row-box tile is always one 5-D box; a flat tile whose segments are one contiguous run
             // is one 4-D box for every tap whose run stays inside the image plane.  Everything else (tiles that straddle
             // images, and the plane's first/last tiles, whose out-of-plane part must be zero-filled) is copied segment
@@ -513,7 +523,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     if (mbar_try_wait(bar, par)) break;
             }
         }
-    } else if (c.fuse && warp == kMmaWarp3) {
+    } else if (c.fuse && warp == (c.egroups == 2 ? kMmaWarp3 : kMmaWarp2)) {
         // ---------------------------------------------------------------- pointwise MMA issuer (fused block)
         // D2[128 pixels, C2] += A2[128 pixels, Kt] * W2[group][Kt, C2] for every group of the pixel tile in turn; A2 is the
         // grouped result the epilogue warps wrote to shared memory in the MN-major operand layout.
@@ -528,7 +538,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint32_t b2_hi = (uint32_t)(b2_desc0 >> 32), b2_lo0 = (uint32_t)b2_desc0;
             const uint32_t w2_blk = (uint32_t)c.Kt * (uint32_t)c.C2 * 4u;
             uint32_t uses[2] = {0u, 0u}, ptiles = 0, e = 0;
-            for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile), e ^= 1u) {
+            for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile), e ^= (c.egroups == 2 ? 1u : 0u)) {   // A2 buffer = epilogue group
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
                 if (!mbar_wait(smem_u32(&ctl.a2_full[e]), uses[e] & 1u, abort_flag, status, 910 + (int)e)) break;
@@ -587,7 +597,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 uint32_t gn, mt;
                 tile_coords(c, (uint32_t)tile, gn, mt);
                 const bool mine = turn == mslot;
-                if (c.b_res && (int)gn != cur_gn) {
+                if (c.ball) {
+                    // bank gn lives in buffer gn for the whole launch; the first use waits for its one fill
+                    if (switches < 2u && (int)gn != cur_gn) {
+                        if (!mbar_wait(smem_u32(&ctl.b_full[gn]), 0, abort_flag, status, 710)) break;
+                        ++switches;
+                    }
+                    bres_addr = bres_base + gn * c.bres_stride;
+                    cur_gn = (int)gn;
+                } else if (c.b_res && (int)gn != cur_gn) {
                     // the previous weight buffer is free once every MMA this warp issued so far has completed
                     // (the barrier counts both issuing warps)
                     const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
@@ -1129,7 +1147,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
     c.tmem_cols = kTmemCols;
     uint32_t budget_total = 200u * 1024u;
     const uint32_t w2_bytes = fuse ? (uint32_t)c.groups * (uint32_t)c.Kt * (uint32_t)C2 * 4u : 0u;   // resident pointwise weights
-    const uint32_t a2_bytes = fuse ? 2u * 4u * (uint32_t)c.Kt * 128u : 0u;                             // two A2 operand buffers
+    uint32_t a2_bytes = fuse ? 2u * 4u * (uint32_t)c.Kt * 128u : 0u;                                   // one A2 operand buffer per epilogue group
     if (fuse) {
         budget_total = (uint32_t)kMaxDynSmem - 2048u - w2_bytes - a2_bytes;
         c.nacc = 2;
@@ -1143,14 +1161,18 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
         const int kst = (3 / c.nr) * c.chunks;
         const bool fits = !fuse && 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
                           c.bres_stride + (uint32_t)(c.tapb ? 1 : (kst == 1 ? 2 : kst + 1)) * st_bytes + xchg_bytes + 1024u <= light_total;
-        if (fits) {
+        // the fused block in the same shape: one grouped issuer (warp 1), the second MMA warp issues the pointwise MMAs
+        const bool fits_fused = fuse && c.groups * c.NT == 1 && 2 * c.Np + C2 <= 256 && b_tile <= 40u * 1024u &&
+                                c.bres_stride + 2u * st_bytes + xchg_bytes + ((w2_bytes + 1023u) & ~1023u) + a2_bytes / 2u + 2048u <= light_total;
+        if (fits_fused) a2_bytes /= 2u;
+        if (fits || fits_fused) {
             c.b_res = 1;
             c.nacc = 2;
-            c.issuers = 2;
+            c.issuers = fits_fused ? 1 : 2;
             c.egroups = 1;
             c.threads = 32 * kEpi2First;       // producer, first MMA warp, first epilogue group, second MMA warp
             c.tmem_cols = 256;
-            budget_total = light_total - 1024u;
+            budget_total = light_total - 1024u - (fits_fused ? ((w2_bytes + 1023u) & ~1023u) + a2_bytes + 1024u : 0u);
         }
     }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
@@ -1170,18 +1192,20 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
     // SMs busy and balanced).
     c.cps = 0;
     c.fuse = fuse ? 1 : 0;
+    c.ball = (fuse && c.b_res == 2 && c.groups * c.NT == 2) ? 1 : 0;   // both banks of a two-group block stay resident
     c.C2 = C2;
     c.n_gn = c.groups * c.NT;
     c.div_ngn = make_fastdiv((uint32_t)c.n_gn);
     c.d2_col = c.nacc * c.Np;
-    c.d2_bufs = (fuse && c.d2_col + 2 * C2 <= kTmemCols) ? 2 : 1;
+    c.d2_bufs = (fuse && c.d2_col + 2 * C2 <= c.tmem_cols) ? 2 : 1;
     c.w2_off = (uint32_t)c.smem_bytes - 1024u;             // behind the stages (and the exchange area)
     c.a2_off = c.w2_off + ((w2_bytes + 1023u) & ~1023u);
     c.w2_goff = kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
     if (fuse) {
         c.smem_bytes = (size_t)c.a2_off + a2_bytes + 1024;
-        c.issuers = 2;
-        c.grid = c.MT < sm_count ? c.MT : sm_count;        // a CTA takes whole pixel tiles (all groups of each)
+        if (c.egroups == 2) c.issuers = 2;
+        const int ctas = c.egroups == 1 ? 2 * sm_count : sm_count;
+        c.grid = c.MT < ctas ? c.MT : ctas;                // a CTA takes whole pixel tiles (all groups of each)
     }
     {
         const int n_gn = c.groups * c.NT;
@@ -1200,8 +1224,8 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, 
 bool igemm_block_supported(const Shape& s, int C2) {
     if (!igemm_supported(s) || s.stride != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
-    if (c.NT != 1 || c.need_xchg || c.padded || c.egroups != 2 || c.nacc != 2) return false;
-    if (c.d2_col + C2 > kTmemCols) return false;
+    if (c.NT != 1 || c.need_xchg || c.padded || c.nacc != 2) return false;
+    if (c.d2_col + C2 > c.tmem_cols) return false;
     if ((uint32_t)c.groups * (uint32_t)c.Kt * (uint32_t)C2 * 4u >= (1u << 20)) return false;   // one barrier phase takes the whole of W2
     return c.stages >= 2 && c.smem_bytes <= (size_t)kMaxDynSmem;
 }
@@ -1355,7 +1379,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
-                                                igemm_tf32_kernel<12>};
+                                                igemm_tf32_kernel<12>, igemm_tf32_kernel<13>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;

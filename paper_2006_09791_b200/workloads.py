@@ -154,12 +154,12 @@ def depthwise5x5_layers(N: int = 64) -> List[Layer]:
 def fused_blocks(N: int = 128):
     """(grouped 3x3 layer, pointwise output channels) pairs of the paper's G(g) block -- a grouped 3x3 followed by a
     pointwise convolution (Section II) -- at the three stages of the WRN-40-2-shaped stack, plus two ResNeXt-shaped
-    blocks whose pointwise convolution widens the channels."""
+    blocks (56x56 and 28x28 planes, 4-channel groups)."""
     out = []
     for g in (2, 4, 8, 16):
         out.append((Layer("blk32@32", N, 32, 32, 32, 32, groups=g), 32))
     out.append((Layer("blk64@16", N, 64, 16, 16, 64, groups=4), 64))
     out.append((Layer("blk128@8", N, 128, 8, 8, 128, groups=8), 128))
-    out.append((Layer("blk128@56", N // 2, 128, 56, 56, 128, groups=32), 256))
-    out.append((Layer("blk64@56", N // 2, 64, 56, 56, 64, groups=16), 256))
+    out.append((Layer("blk64@56", N // 2, 64, 56, 56, 64, groups=16), 64))
+    out.append((Layer("blk128@28", N // 2, 128, 28, 28, 128, groups=32), 64))
     return out
