@@ -218,7 +218,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball;
 };
-constexpr int kFamilies = 14;
+constexpr int kFamilies = 15;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -234,6 +234,7 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes with halo stages
          : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
          : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes, two CTAs per SM
+         : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1}     // fused block, row boxes, two resident banks
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1379,7 +1380,8 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
-                                                igemm_tf32_kernel<12>, igemm_tf32_kernel<13>};
+                                                igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
+                                                igemm_tf32_kernel<14>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
