@@ -182,8 +182,10 @@ int gconv_forward_host_static(gconv_desc_t desc, const float *x_host, const void
  * gconv_block_supported  1 if the pair (descriptor, C2) can run fused, else 0: 3x3, pad 1, stride 1, dilation 1,
  *                        W a multiple of 4 and at most 62 or equal to 64 wide planes only where the grouped kernel
  *                        needs no edge exchange, merged group width a multiple of 8 with at most 64 filters per
- *                        group, C2 a multiple of 16 with 2 * 3 * (filters per merged group) + C2 <= 512, and the
- *                        resident pointwise weights (C_out * C2 * 4 bytes) must leave room for two input stages.
+ *                        group, C2 a multiple of 16 from 16 to 256 with 2 * 3 * (filters per merged group) + C2 <= 512,
+ *                        and the resident pointwise weights (C_out * C2 * 4 bytes) must leave room for two input
+ *                        stages.  "Supported" is not "faster than two launches": fusing pays on large planes
+ *                        (32x32 and up), small planes with several groups per pixel tile run faster unfused.
  * gconv_block_packed_bytes  size of the packed buffer holding both weight tensors (0 if unsupported).
  * gconv_block_pack_weights  w_ochw device fp32 [C_out, C_in/groups, 3, 3]; w2 device fp32 [C2, C_out]; both rounded
  *                        to TF32 while packing; asynchronous on `stream`.
