@@ -292,6 +292,91 @@ dw5_stream_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, con
     if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 }
 
+// 5x5, stride 1: U5 output rows per block, the raw input rows of the next two blocks in flight during the block's
+// math (four 16-byte loads per thread).  An input row feeds five output rows, so its eight-column window (own four
+// columns plus two from each neighbouring lane) is built once, when the row enters the block, and kept in registers:
+// four shuffles per input row instead of twenty.
+constexpr int U5 = 2;   // output rows per block of the 5x5 kernel
+constexpr int D5 = 4;   // raw rows in flight beyond the current block
+template <int VEC>
+__global__ void __launch_bounds__(256, 2)
+dw5_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
+                     float* __restrict__ y, Status* status, uint32_t tag) {
+    const uint32_t tag_seen = __ldg(packed);
+    const float* __restrict__ wpk = reinterpret_cast<const float*>(packed + kHeaderBytes / 4);
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int sub = lane / c.XQ;
+    const int xq = lane - sub * c.XQ;
+    const uint32_t item = warp_global * (uint32_t)c.subs + (uint32_t)sub;
+    const bool live = (sub < c.subs) && (item < c.items);
+    uint32_t plane_idx = 0, chunk = 0;
+    c.div_chunks.divmod(live ? item : 0u, plane_idx, chunk);
+    const int ch = (int)(plane_idx % (uint32_t)s.C_in);
+    const float* __restrict__ xp = x + (size_t)plane_idx * s.H * s.W;
+    float* __restrict__ yp = y + (size_t)plane_idx * s.H * s.W;
+    const int col = xq * 4;
+    const int p0 = (int)chunk * c.RH;
+    const int p1 = min(p0 + c.RH, s.H);
+    const bool has_l = xq > 0, has_r = xq < c.XQ - 1;
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // rows p0-2 .. p0+U5+1 fill the first block's windows, rows up to p0+U5+1+D5 wait in the queue; row h is needed
+    // only if it feeds an output row of this strip (h <= p1+1)
+    float4 first[U5 + 4], queue[D5];
+#pragma unroll
+    for (int j = 0; j < U5 + 4; ++j) first[j] = live ? ldrow<VEC>(xp, p0 - 2 + j, s.H, s.W, col) : z4;
+#pragma unroll
+    for (int j = 0; j < D5; ++j) {
+        const int h = p0 + U5 + 2 + j;
+        queue[j] = (live && h <= p1 + 1) ? ldrow<VEC>(xp, h, s.H, s.W, col) : z4;
+    }
+    float w[5][5];
+#pragma unroll
+    for (int i = 0; i < 25; ++i) w[i / 5][i % 5] = live ? __ldg(wpk + (size_t)ch * 25 + i) : 0.f;
+    auto widen = [&](const float4 v, float (&o)[8]) {   // every lane runs the shuffles; `live` only gates memory traffic
+        const float l0 = __shfl_up_sync(0xffffffffu, v.z, 1), l1 = __shfl_up_sync(0xffffffffu, v.w, 1);
+        const float r0 = __shfl_down_sync(0xffffffffu, v.x, 1), r1 = __shfl_down_sync(0xffffffffu, v.y, 1);
+        o[0] = has_l ? l0 : 0.f;
+        o[1] = has_l ? l1 : 0.f;
+        o[2] = v.x; o[3] = v.y; o[4] = v.z; o[5] = v.w;
+        o[6] = has_r ? r0 : 0.f;
+        o[7] = has_r ? r1 : 0.f;
+    };
+    float win[U5 + 4][8];                              // input rows p-2 .. p+U5+1 of the current block
+#pragma unroll
+    for (int j = 0; j < U5 + 4; ++j) widen(first[j], win[j]);
+    for (int p = p0; p < p0 + c.RH; p += U5) {         // warp-uniform trip count
+        float4 fresh[U5];
+#pragma unroll
+        for (int j = 0; j < U5; ++j) {
+            const int h = p + U5 + 2 + D5 + j;
+            fresh[j] = (live && h <= p1 + 1) ? ldrow<VEC>(xp, h, s.H, s.W, col) : z4;
+        }
+#pragma unroll
+        for (int j = 0; j < U5; ++j) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < 5; ++r)
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int t = 0; t < 5; ++t) acc[q] = fmaf(win[j + r][q + t], w[r][t], acc[q]);
+            if (live && p + j < p1 && tag_seen == tag) strow<VEC>(yp + (size_t)(p + j) * s.W + col, col, s.W, acc);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) win[j][i] = win[j + U5][i];
+#pragma unroll
+        for (int j = 0; j < U5; ++j) widen(queue[j], win[4 + j]);
+#pragma unroll
+        for (int j = 0; j + U5 < D5; ++j) queue[j] = queue[j + U5];
+#pragma unroll
+        for (int j = 0; j < U5; ++j) queue[D5 - U5 + j] = fresh[j];
+    }
+    if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
+}
+
 }  // namespace
 
 bool dw_supported(const Shape& s) {
@@ -308,10 +393,12 @@ DwCfg dw_config(const Shape& s, int sm_count) {
     c.XQ = s.stride == 1 ? (s.W + 3) / 4 : (s.W + 7) / 8;
     c.subs = 32 / c.XQ;
     // rows per thread: long strips amortise the two halo rows, short ones give more parallelism; aim for
-    // at least ~6 waves of 1024 threads per SM
+    // at least ~6 waves of 1024 threads per SM.  5x5: four halo rows per strip and 25 FMAs per output make the strip
+    // length matter more than the thread count (measured): split only below ~0.4 waves.
     const long long planes = (long long)s.N * s.C_in;
+    const long long want = s.KH == 5 ? 410LL * sm_count : 6LL * 1024 * sm_count;
     int rh = s.H_out;
-    while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < 6LL * 1024 * sm_count) rh = (rh + 1) / 2;
+    while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < want) rh = (rh + 1) / 2;
     rh = ((rh + U - 1) / U) * U;
     c.RH = rh;
     c.chunks = (s.H_out + rh - 1) / rh;
@@ -332,7 +419,7 @@ cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float
     do { \
         if (vec == 4) KERNEL(4); else if (vec == 2) KERNEL(2); else KERNEL(0); \
     } while (0)
-#define GCONV_DW5_S1(V) dw5_stream_kernel<V, 1><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
+#define GCONV_DW5_S1(V) dw5_stream_s1_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
 #define GCONV_DW5_S2(V) dw5_stream_kernel<V, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
 #define GCONV_DW3_S1(V) dw_stream_s1_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
 #define GCONV_DW3_S2(V) dw_stream_s2_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)

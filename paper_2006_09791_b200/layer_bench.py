@@ -1,7 +1,7 @@
 """Time one grouped-convolution layer through the C ABI (also the entry used for ncu captures).
 
     python -m paper_2006_09791_b200.layer_bench --cin 32 --cout 32 --hw 32 --groups 1 --n 128 \
-        [--stride 1] [--variant auto|generic|tiled|igemm] [--reps 20] [--bufs 0] [--c2 C2]
+        [--stride 1] [--k 3] [--variant auto|generic|tiled|igemm] [--reps 20] [--bufs 0] [--c2 C2]
 
 With --c2 the fused block runs instead (this grouped 3x3 followed by a pointwise convolution to C2 channels,
 gconv_block_forward); bytes and FLOPs then count x, y2 and both contractions.
@@ -34,6 +34,7 @@ def main():
     ap.add_argument("--groups", type=int, default=1)
     ap.add_argument("--n", type=int, default=1)
     ap.add_argument("--stride", type=int, default=1)
+    ap.add_argument("--k", type=int, default=3, help="square filter size, pad = k // 2")
     ap.add_argument("--variant", default="auto", choices=sorted(VARIANTS))
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -41,12 +42,12 @@ def main():
     ap.add_argument("--c2", type=int, default=0)
     a = ap.parse_args()
     gbuild.build()
-    L = Layer("layer", a.n, a.cin, a.hw, a.w or a.hw, a.cout or a.cin, stride=a.stride, groups=a.groups)
+    L = Layer("layer", a.n, a.cin, a.hw, a.w or a.hw, a.cout or a.cin, a.k, a.k, a.stride, a.k // 2, 1, a.groups)
     dev = torch.device("cuda:0")
     y_elems = L.N * a.c2 * L.H_out * L.W_out if a.c2 else L.y_elems
     per = 4 * (L.x_elems + y_elems)
     nbuf = a.bufs or max(2, -(-(2 * 126 * 2 ** 20 + (64 << 20)) // per))
-    x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 7)
+    x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.groups, 7)
     xs = [torch.from_numpy(x0).to(dev).repeat(-(-L.N // x0.shape[0]), 1, 1, 1)[:L.N].contiguous() for _ in range(nbuf)]
     ys = [torch.empty(y_elems, dtype=torch.float32, device=dev) for _ in range(nbuf)]
     d = gconv.gconv_desc_create(*L.desc_args())
