@@ -129,3 +129,51 @@ def test_more_than_2_to_31_elements():
             torch.cuda.empty_cache()
         finally:
             gconv.gconv_desc_destroy(d)
+
+
+def _fused_blocks():
+    from paper_2006_09791_b200.workloads import fused_blocks
+    return fused_blocks()
+
+
+@pytest.mark.parametrize("idx", range(len(_fused_blocks())))
+def test_fused_blocks_at_bench_batch(idx):
+    """The fused grouped 3x3 + pointwise blocks the bench times, at its batch, back to back (two launches, the second a
+    CUDA-graph replay on odd rows).  Sampled images are checked in full: the oracle's grouped convolution of the image,
+    rounded to fp32 (the kernel keeps the intermediate in fp32), then its 1x1 convolution."""
+    L, C2 = _fused_blocks()[idx]
+    dev = torch.device("cuda:0")
+    x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(81, idx), L.x_dist)
+    _, w2 = synth.make_layer_tensors(1, L.C_out, 1, 1, C2, 1, 1, 1, synth.layer_seed(82, idx))
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_block_supported(d, C2)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            xd = torch.from_numpy(x).to(dev)
+            wp = torch.empty(gconv.gconv_block_packed_bytes(d, C2) // 4, dtype=torch.float32, device=dev)
+            y2 = torch.full((L.N * C2 * L.H * L.W,), float("nan"), dtype=torch.float32, device=dev)
+            scratch = torch.empty_like(y2)
+            gconv.gconv_block_pack_weights(d, C2, torch.from_numpy(w).to(dev), torch.from_numpy(w2.reshape(C2, L.C_out)).to(dev), wp, s)
+            gconv.gconv_block_forward(d, C2, xd, wp, scratch, s)
+            if idx % 2 == 1:
+                s.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=s):
+                    gconv.gconv_block_forward(d, C2, xd, wp, scratch, s)
+                    gconv.gconv_block_forward(d, C2, xd, wp, y2, s)
+                graph.replay()
+            else:
+                gconv.gconv_block_forward(d, C2, xd, wp, y2, s)
+            s.synchronize()
+        assert gconv.gconv_last_status(d, s) == gconv.GCONV_OK
+        got = y2.cpu().numpy().reshape(L.N, C2, L.H, L.W)
+        assert np.all(np.isfinite(got))
+        tol = gconv.VARIANT_TOLERANCE[gconv.GCONV_VARIANT_IGEMM_TF32]
+        for n in sorted({0, L.N - 1, (7 * idx + 3) % L.N}):
+            y1 = oracle.gconv_ref(x[n:n + 1], w, 1, 1, 1, L.groups, threads=16).astype(np.float32)
+            ref = oracle.gconv_ref(y1, w2, 1, 0, 1, 1, threads=16)[0]
+            err = np.max(np.abs(got[n].astype(np.float64) - ref)) / np.max(np.abs(ref))
+            assert err <= tol, (L.name, L.groups, C2, n, err)
+    finally:
+        gconv.gconv_desc_destroy(d)
