@@ -120,7 +120,8 @@ int gconv_pack_weights(gconv_desc_t desc, const float *w_ochw, void *w_packed, v
  *   x_nchw    device, fp32 [N, C_in, H, W], read only; must not overlap y.
  *   w_packed  device, produced by gconv_pack_weights on a descriptor of the same shape and variant.
  *   y_nchw    device, fp32 [N, C_out, H_out, W_out], every element written.
- * For layers whose width is not a multiple of 4 the tensor-core variant computes on a zero-padded copy of x that
+ * For some layers whose width is not a multiple of 4 (gconv_forward_launches reports 2 for them: wide groups,
+ * stride 2 on such planes, large 7x7 layers) the tensor-core variant computes on a zero-padded copy of x that
  * it keeps in a device scratch buffer owned by the descriptor: that buffer is allocated (cudaMalloc) by the first
  * gconv_forward of such a descriptor -- make that call outside any stream capture -- and freed by
  * gconv_desc_destroy; two concurrent forwards of ONE such descriptor would race on it.

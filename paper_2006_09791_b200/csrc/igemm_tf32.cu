@@ -50,6 +50,7 @@ constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the fir
 constexpr int kEpi2First = kMmaWarp2 + 1;    // first warp of the second epilogue group
 constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issuing warps (used when four accumulators fit)
 constexpr int kThreads = 32 * (kMmaWarp3 + 2);
+constexpr int kSoftWarps = 4;        // copy warps of the software producer (light launch shape only): warps kEpi2First ...
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 // Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
@@ -89,6 +90,19 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// Non-blocking probe (try_wait may suspend the thread for a hardware time limit while the phase is incomplete).
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -216,30 +230,32 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball;
+        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft;
 };
-constexpr int kFamilies = 15;
+constexpr int kFamilies = 17;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0}     // row boxes of one segment, narrow groups
-         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
-         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes with halo stages
-         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
-         : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0}     // fused block, 32-wide planes, two CTAs per SM
-         : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1}     // fused block, row boxes, two resident banks
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0,  0}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0,  0}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0,  0}     // row boxes of one segment, narrow groups
+         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0}     // fused block, 32-wide planes with halo stages
+         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1,  0}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
+         : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0}     // fused block, 32-wide planes, two CTAs per SM
+         : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0}     // fused block, row boxes, two resident banks
+         : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1}     // copy-warp producer (14x14, 7x7 planes), tap blocks
+         : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1}     // copy-warp producer, one stage per tap
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball) X(soft)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -252,7 +268,8 @@ static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
 
 __device__ __forceinline__ void
 igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& s, const IgemmCfg& c,
-                const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag) {
+                const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag,
+                const float* __restrict__ x) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
     static_assert(sizeof(SharedCtl) <= 1024, "control block must leave 226 KB of dynamic shared memory");
@@ -278,7 +295,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         const int t = (int)threadIdx.x - 64;
         if (t >= 0 && t < 8) {
             if (t < c.stages) {
-                mbar_init(smem_u32(&ctl.full[t]), 1);
+                mbar_init(smem_u32(&ctl.full[t]), c.soft ? (uint32_t)kSoftWarps : 1u);
                 mbar_init(smem_u32(&ctl.empty[t]), 1);
             }
         } else if (t >= 8 && t < 8 + kMaxAcc) {
@@ -401,7 +418,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2 instead
         // of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
         // Pass 1 is the real one.
-        for (int pass = 0; pass < 2 && ok; ++pass) {
+        for (int pass = (c.soft ? 1 : 0); pass < 2 && ok; ++pass) {
         const bool pf = pass == 0;
         if (!pf) {
             asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
@@ -417,6 +434,21 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const int g = (int)gq;
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
             const bool switch_b = !pf && c.b_res && !c.ball && (int)gn != cur_gn;
+            if (c.soft) {
+                // the copy warps stage the input; this warp only brings the resident weights of a new (group, filter tile)
+                if (switch_b) {
+                    const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
+                    if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&ctl.b_full[bb]);
+                    if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
+                    __syncwarp();
+                    for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                        bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
+                    cur_gn = (int)gn;
+                    ++switches;
+                }
+                continue;
+            }
             // Whole-tile copies: a row-box tile is always one 5-D box; a flat tile whose segments are one contiguous run
             // is one 4-D box for every tap whose run stays inside the image plane.  Everything else (tiles that straddle
             // images, and the plane's first/last tiles, whose out-of-plane part must be zero-filled) is copied segment
@@ -560,6 +592,88 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 }
             }
         }
+    } else if (c.soft && warp >= kEpi2First) {
+        // ---------------------------------------------------------------- software producer (copy warps)
+        // Widths TMA cannot address (rows that are not a multiple of 16 bytes: 14, 7, ...): the kernel computes on a
+        // virtual zero-padded plane (s.H x s.W, a power-of-two width that divides 32) and these warps build the
+        // stages themselves -- cp.async of 8 bytes (even widths) or 4 bytes from the real rows into exactly the
+        // shared-memory image TMA would have written (32-pixel blocks, 128-byte row per channel, 32-byte chunks
+        // XOR-swizzled by the channel), zero-size copies for the pad columns, the rows outside the plane and the images
+        // past the batch.  Warp j of the four owns segment j of every four-segment block.  A stage is handed to the
+        // tensor core one stage late: after issuing the next stage's copies the warp waits for its own copies of the
+        // previous one (cp.async groups), makes them visible to the async proxy and arrives on the stage's barrier.
+        // Before it blocks on a stage that is still being read it hands over what it holds (a ring of one stage
+        // would otherwise wait for itself).
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int pw = warp - kEpi2First;
+        const bool pairs = (c.Wv & 1) == 0;                 // two pixels per copy
+        const int u = pairs ? (lane & 15) : lane;           // copy unit inside the 32-pixel segment
+        const int kfirst = pairs ? (lane >> 4) : 0, kstep = pairs ? 2 : 1;
+        const int wshift = __ffs(s.W) - 1;
+        const size_t plane = (size_t)c.Hv * (size_t)c.Wv;
+        const uint32_t unit_off = pairs ? ((uint32_t)(u >> 2) << 5) + (uint32_t)(u & 3) * 8u : ((uint32_t)(u >> 3) << 5) + (uint32_t)(u & 7) * 4u;
+        const uint32_t unit_chunk = pairs ? (uint32_t)(u >> 2) : (uint32_t)(u >> 3);
+        const uint32_t unit_in = pairs ? (uint32_t)(u & 3) * 8u : (uint32_t)(u & 7) * 4u;
+        (void)unit_off;
+        uint32_t it = 0;
+        int stage = 0, prev_stage = 0;
+        uint32_t ph = 0;
+        bool ok = true, pending = false;                    // pending: prev_stage's copies are issued but not handed over
+        auto hand_over = [&](bool all) {
+            if (all) asm volatile("cp.async.wait_group 0;" ::: "memory");
+            else asm volatile("cp.async.wait_group 1;" ::: "memory");   // every group but the newest
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.full[prev_stage]));
+        };
+        for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile)) {
+            uint32_t gn, mt;
+            tile_coords(c, (uint32_t)tile, gn, mt);
+            uint32_t gq = gn, ntq = 0;
+            if (c.NT > 1) c.div_nt.divmod(gn, gq, ntq);
+            uint32_t n, i;
+            c.div_spi.divmod(mt * 4u + (uint32_t)pw, n, i);
+            const bool img_ok = (int)n < s.N;
+            int ch = 0, r = 0;
+            for (int ks = 0; ks < kstages; ++ks, ++it) {
+                if (it >= (uint32_t)c.stages) {
+                    const uint32_t bar = smem_u32(&ctl.empty[stage]);
+                    if (!__all_sync(0xffffffffu, mbar_test_wait(bar, ph ^ 1) ? 1 : 0)) {
+                        if (pending) { hand_over(true); pending = false; }
+                        if (!mbar_wait_warp(bar, ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                    }
+                }
+                const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
+                const float* xg = x + ((size_t)(img_ok ? n : 0u) * s.C_in + (size_t)((int)gq * c.Cg + ch * c.CK)) * plane;
+                const int ntb = c.tapb ? 3 : 1;
+                for (int tb = 0; tb < ntb; ++tb) {
+                    const int tap = c.tapb ? tb : r;
+                    const int f = (int)i * c.seg_fstep + (tap - 1) * s.W + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
+                    const int row = f >> wshift, col = f & (s.W - 1);
+                    const bool valid = img_ok && f >= 0 && row < c.Hv && col < c.Wv;
+                    const float* src = valid ? xg + (size_t)row * c.Wv + col : x;
+                    const uint32_t nbytes = valid ? (pairs ? 8u : 4u) : 0u;
+                    const uint32_t dseg = a_dst + (uint32_t)(tb * 4 + pw) * seg_bytes + unit_in;
+                    if (pairs) {
+                        for (int k = kfirst; k < c.CK; k += kstep)
+                            asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dseg + (uint32_t)k * 128u + ((unit_chunk ^ ((uint32_t)k & 3u)) << 5)),
+                                         "l"(src + (size_t)k * plane), "r"(nbytes) : "memory");
+                    } else {
+                        for (int k = kfirst; k < c.CK; k += kstep)
+                            asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dseg + (uint32_t)k * 128u + ((unit_chunk ^ ((uint32_t)k & 3u)) << 5)),
+                                         "l"(src + (size_t)k * plane), "r"(nbytes) : "memory");
+                    }
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                if (pending) hand_over(false);
+                pending = true;
+                prev_stage = stage;
+                if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
+                if (++stage == c.stages) { stage = 0; ph ^= 1; }
+            }
+        }
+        if (pending && ok) hand_over(true);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp == 1 || warp == kMmaWarp2 || warp >= kMmaWarp3) {
         // ---------------------------------------------------------------- MMA issuers
         // Two warps issue alternate tiles (each owns one TMEM buffer), so the barrier waits and descriptor
@@ -849,12 +963,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     }
 }
 
+// (the copy-warp families run two 480-thread CTAs per SM: at most 68 registers per thread)
 template <int F>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(family(F).soft == 1 ? 32 * (kEpi2First + kSoftWarps) : kThreads, family(F).soft == 1 ? 2 : 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xmap4, const Shape s_in,
-                  const IgemmCfg c_in, const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag) {
+                  const IgemmCfg c_in, const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag,
+                  const float* __restrict__ x) {
     if constexpr (F == 0) {
-        igemm_tf32_body(xmap, xmap4, s_in, c_in, packed, y, status, tag);
+        igemm_tf32_body(xmap, xmap4, s_in, c_in, packed, y, status, tag, x);
     } else {
         constexpr Family fam = family(F);
         IgemmCfg c = c_in;
@@ -863,7 +979,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         GCONV_FAMILY_FIELDS(GCONV_FIX)
 #undef GCONV_FIX
         if constexpr (fam.stride >= 0) s.stride = fam.stride;
-        igemm_tf32_body(xmap, xmap4, s, c, packed, y, status, tag);
+        igemm_tf32_body(xmap, xmap4, s, c, packed, y, status, tag, x);
     }
 }
 
@@ -1006,7 +1122,8 @@ bool igemm_supported(const Shape& s) {
 
 size_t igemm_scratch_bytes(const Shape& s) {
     const IgemmGeom ge = igemm_geom(s);
-    return ge.padded ? sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp : 0;
+    if (!ge.padded || igemm_config(s, kLayoutSMs).soft) return 0;   // copy warps read the real rows: no padded copy
+    return sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp;
 }
 
 static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
@@ -1176,6 +1293,16 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
             budget_total = light_total - 1024u - (fits_fused ? ((w2_bytes + 1023u) & ~1023u) + a2_bytes + 1024u : 0u);
         }
     }
+    // Software producer: a width TMA cannot address whose padded plane is a whole number of segments, in the light
+    // shape.  The copy warps read the real rows, so there is no padded copy of x and no extra launch.
+    // Odd widths copy four bytes at a time, which only pays while the layer is small (measured: 7x7 planes, 3 MB of x
+    // 22 % faster, 13 MB 12 % slower than the padded copy); even widths copy eight and always pay.
+    const bool soft_pays = (s_true.W % 2 == 0) || (size_t)s_true.N * s_true.C_in * s_true.H * s_true.W * 4u <= (8u << 20);
+    c.soft = (ge.padded && c.seg_mode && c.egroups == 1 && !fuse && soft_pays) ? 1 : 0;
+    if (c.soft) {
+        c.padded = 0;
+        c.threads += 32 * kSoftWarps;
+    }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
     c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
     const uint32_t budget = budget_total - (uint32_t)c.b_res * c.bres_stride - xchg_bytes;
@@ -1319,6 +1446,11 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
         s.H = ge.Hp;
         s.W = ge.Wp;
         x = scratch;
+    } else if (c.soft) {
+        // the kernel walks the virtual padded plane; its copy warps read the real rows of x (the tensor maps go unused)
+        const IgemmGeom ge = igemm_geom(s_true);
+        s.H = ge.Hp;
+        s.W = ge.Wp;
     }
     EncodeTiledFn encode = get_encode_fn();
     if (encode == nullptr) return cudaErrorNotSupported;
@@ -1337,7 +1469,9 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     IgemmCfg cfg = c;
     CUtensorMap xmap4 = xmap;
     cfg.fast4 = 0;
-    if (c.rowbox) {
+    if (c.soft) {
+        // no second map
+    } else if (c.rowbox) {
         // (column, channel, row segment, row, image); the segment axis steps (W - 32) columns
         const cuuint64_t dims5[5] = {(cuuint64_t)s.W, (cuuint64_t)s.C_in, (cuuint64_t)c.SR, (cuuint64_t)s.H, (cuuint64_t)s.N};
         const cuuint64_t strides5[4] = {HW * 4, c.SR == 2 ? (cuuint64_t)(s.W - 32) * 4 : 128, (cuuint64_t)s.W * 4,
@@ -1375,13 +1509,14 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
         else
             xmap4 = xmap;
     }
-    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const Shape, const IgemmCfg, const uint32_t*, float*, Status*, uint32_t);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const Shape, const IgemmCfg, const uint32_t*, float*, Status*, uint32_t,
+                              const float*);
     static const KernelFn kernels[kFamilies] = {igemm_tf32_kernel<0>, igemm_tf32_kernel<1>, igemm_tf32_kernel<2>,
                                                 igemm_tf32_kernel<3>, igemm_tf32_kernel<4>, igemm_tf32_kernel<5>,
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
-                                                igemm_tf32_kernel<14>};
+                                                igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
@@ -1404,7 +1539,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     lc.attrs = attr;
     lc.numAttrs = 1;
     return cudaLaunchKernelEx(&lc, kernels[fam], xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
-                              C2 > 0 ? block_tag(s_true, C2) : pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32));
+                              C2 > 0 ? block_tag(s_true, C2) : pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32), x);
 }
 
 

@@ -99,6 +99,29 @@ def test_large_rowbox_shapes(cfg):
     check_layer(Layer("rowbox", *cfg), seed=11)
 
 
+# Widths whose rows are not a multiple of 16 bytes, in the configurations where copy warps (cp.async) build the stages
+# instead of TMA: even widths (8-byte copies) and odd ones (4-byte), padded widths 8, 16 and 32, planes that end inside
+# a tile, batches that end inside a tile, many tiles per CTA, several groups per CTA, stride 2 on 7x7 planes.
+COPY_WARP_SHAPES = [
+    (5, 32, 14, 14, 32, 3, 3, 1, 1, 1, 4), (9, 64, 7, 7, 64, 3, 3, 1, 1, 1, 2), (2, 16, 17, 30, 16, 3, 3, 1, 1, 1, 2),
+    (3, 24, 10, 6, 24, 3, 3, 1, 1, 1, 3), (4, 32, 15, 15, 32, 3, 3, 1, 1, 1, 1), (2, 8, 9, 31, 16, 3, 3, 1, 1, 1, 1),
+    (7, 32, 7, 7, 32, 3, 3, 2, 1, 1, 4), (300, 64, 14, 14, 64, 3, 3, 1, 1, 1, 2), (40, 512, 14, 14, 512, 3, 3, 1, 1, 1, 32),
+    (33, 256, 7, 7, 256, 3, 3, 1, 1, 1, 8), (1, 8, 5, 7, 8, 3, 3, 1, 1, 1, 1), (6, 48, 13, 14, 96, 3, 3, 1, 1, 1, 6),
+]
+
+
+@pytest.mark.parametrize("cfg", COPY_WARP_SHAPES)
+def test_copy_warp_producer_shapes(cfg):
+    L = Layer("copywarp", *cfg)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32
+        assert gconv.gconv_forward_launches(d) == 1          # no padding pass: the copy warps read the real rows
+    finally:
+        gconv.gconv_desc_destroy(d)
+    check_layer(L, seed=23)
+
+
 @pytest.mark.parametrize("groups", [1, 2, 4, 8, 16])
 def test_wrn_stack_small_batch(groups):
     """Every distinct layer of the WRN-40-2-shaped stack at N = 1 and a ragged N = 3, all variants."""
@@ -185,7 +208,7 @@ def test_depthwise_5x5_network_shapes():
 
 
 @pytest.mark.parametrize("shape", [(16, 32, 32, 32, 4), (8, 64, 16, 16, 2), (24, 128, 8, 8, 8), (6, 64, 28, 28, 1), (4, 16, 56, 56, 16),
-                                   (4, 32, 14, 14, 4), (8, 32, 28, 28, 32), (3, 256, 14, 14, 1)])
+                                   (4, 32, 14, 14, 4), (8, 32, 28, 28, 32), (3, 256, 14, 14, 1), (20, 64, 7, 7, 2)])
 def test_dependent_chain_back_to_back(shape):
     """Five layers launched back to back on one stream, each reading the previous layer's output (the kernels start
     their set-up, weight fetch and an L2 prefetch before the previous kernel has finished, so this is the case that
