@@ -263,7 +263,7 @@ static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     GCONV_FAMILY_FIELDS(GCONV_CHK)
 #undef GCONV_CHK
     if (fam.stride >= 0 && s.stride != fam.stride) return false;
-    return true;
+    return s.dilation == 1;          // every family fixes dilation 1; dilated layers run the generic instantiation
 }
 
 __device__ __forceinline__ void
@@ -362,6 +362,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     const uint32_t bres_base = smem_base;                                // two resident weight buffers (if b_res)
     const uint32_t stage_base = smem_base + (uint32_t)c.b_res * c.bres_stride;   // b_res = number of resident weight buffers
     const int HW = s.H * s.W;
+    const int rstep = s.W * s.dilation;          // flat-pixel distance between vertical taps
     const size_t OHW = (size_t)s.H_out * s.W_out;
 
     if (!tag_ok) {
@@ -477,7 +478,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
                 const int chan = g * c.Cg + ch * c.CK;
-                const int lo = tile_f0 + (r - 1) * s.W - c.wseg * 32;
+                const int lo = tile_f0 + (r - 1) * rstep - c.wseg * 32;
                 const bool box = c.rowbox || c.fast4 == 2 || (c.fast4 == 1 && lo >= 0 && lo + c.nseg * 32 <= HW);
                 if (lane == 0 && pf) {
                     if (box) {
@@ -518,8 +519,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     }
                     __syncwarp();                          // the barrier is armed before any lane's copy can complete on it
                     if (lane < c.nseg) {
-                        if (pf) tma_prefetch_3d(&xmap, my_f + (r - 1) * s.W, chan, my_n);
-                        else tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * s.W, chan, my_n, full);
+                        if (pf) tma_prefetch_3d(&xmap, my_f + (r - 1) * rstep, chan, my_n);
+                        else tma_load_3d(a_dst + (uint32_t)lane * seg_bytes, &xmap, my_f + (r - 1) * rstep, chan, my_n, full);
                     }
                 }
                 if (ks == 0 && switch_b) {
@@ -648,7 +649,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const int ntb = c.tapb ? 3 : 1;
                 for (int tb = 0; tb < ntb; ++tb) {
                     const int tap = c.tapb ? tb : r;
-                    const int f = (int)i * c.seg_fstep + (tap - 1) * s.W + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
+                    const int f = (int)i * c.seg_fstep + (tap - 1) * rstep + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
                     const int row = f >> wshift, col = f & (s.W - 1);
                     const bool valid = img_ok && f >= 0 && row < c.Hv && col < c.Wv;
                     const float* src = valid ? xg + (size_t)row * c.Wv + col : x;
@@ -853,8 +854,9 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             }
             uint32_t prow, q;
             c.div_w.divmod((uint32_t)f, prow, q);
-            const bool use_left = q > 0;
-            const bool use_right = (int)q < s.W - 1;
+            const int dil = s.dilation;                  // horizontal taps sit dil columns away (dil > 1: segment tilings only)
+            const bool use_left = (int)q >= dil;
+            const bool use_right = (int)q + dil < s.W;
             // s.H x s.W is the (possibly padded) plane the kernel computes on; only the first Hv x Wv pixels exist in y
             valid = valid && (int)prow < c.Hv && (int)q < c.Wv;
             int fo = (int)prow * s.W_out + (int)q;       // position in the output plane
@@ -862,8 +864,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
                 fo = (int)(prow >> 1) * s.W_out + (int)(q >> 1);
             }
-            const bool add_up = use_left && lane > 0;
-            const bool add_dn = use_right && lane < 31;
+            const bool add_up = use_left && lane >= dil;
+            const bool add_dn = use_right && lane + dil < 32;
             if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), bph, abort_flag, status, 400 + buf)) break;
             tc_fence_after();
             const uint32_t t0 = tmem_base + buf * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
@@ -902,8 +904,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const float up = __shfl_up_sync(0xffffffffu, d0[j], 1);
-                    const float dn = __shfl_down_sync(0xffffffffu, d2[j], 1);
+                    const float up = __shfl_up_sync(0xffffffffu, d0[j], (unsigned)dil);
+                    const float dn = __shfl_down_sync(0xffffffffu, d2[j], (unsigned)dil);
                     float v = d1[j];
                     if (add_up) v += up;
                     if (add_dn) v += dn;
@@ -979,6 +981,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         GCONV_FAMILY_FIELDS(GCONV_FIX)
 #undef GCONV_FIX
         if constexpr (fam.stride >= 0) s.stride = fam.stride;
+        s.dilation = 1;
         igemm_tf32_body(xmap, xmap4, s, c, packed, y, status, tag, x);
     }
 }
@@ -1110,14 +1113,19 @@ static int igemm_merge(const Shape& s) {
 }
 
 bool igemm_supported(const Shape& s) {
-    if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.pad == 1 && s.dilation == 1)) return false;
+    if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.dilation >= 1 && s.pad == s.dilation)) return false;
+    if (s.dilation > 1 && (s.stride != 1 || s.dilation > 16)) return false;
     const int m = igemm_merge(s);
     if ((s.Cg * m) % 8 != 0 || (s.Kg * m) % 8 != 0) return false;
     const IgemmGeom ge = igemm_geom(s);
     if (ge.Wp > 128) return false;
     if ((long long)ge.Hp * ge.Wp < 32) return false;
     if (s.C_in > 65535 * 8) return false;
-    return igemm_config(s, 148).smem_bytes <= (size_t)kMaxDynSmem;   // the smallest pipeline (two stages) must fit
+    const IgemmCfg c = igemm_config(s, 148);
+    // Dilation: vertical taps are whole-row shifts for any tiling, but the horizontal neighbours dil columns away must
+    // lie in the same 32-pixel segment: segment tilings only (rows that divide 32 pixels).
+    if (s.dilation > 1 && !(c.seg_mode && !c.rowbox && c.nr == 1 && !c.tapb)) return false;
+    return c.smem_bytes <= (size_t)kMaxDynSmem;   // the smallest pipeline (two stages) must fit
 }
 
 size_t igemm_scratch_bytes(const Shape& s) {
@@ -1218,7 +1226,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
         c.nr = 3;
         c.wseg = c.SR;
         c.nseg = 4 + 2 * c.SR;
-    } else if (s.stride == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
+    } else if (s.stride == 1 && s.dilation == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
         c.nr = 3;
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
@@ -1228,7 +1236,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
     // segments, each loaded with its own row shift -- so a tile costs one barrier round trip instead of three.  Only
     // where a tile straddles images anyway (8x8): 16x16 planes keep their one-box-per-tap copies, which are faster.
     c.tapb = 0;
-    if (!fuse && c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
+    if (!fuse && c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && s.dilation == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
         3u * (uint32_t)c.Cg * (uint32_t)c.Np * 4u <= 40u * 1024u) {
         c.tapb = 1;
         c.nr = 3;
@@ -1350,7 +1358,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, 
 
 // ---- fused block: grouped 3x3 followed by a pointwise (1x1, groups = 1) convolution C_out -> C2 ------------------------
 bool igemm_block_supported(const Shape& s, int C2) {
-    if (!igemm_supported(s) || s.stride != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
+    if (!igemm_supported(s) || s.stride != 1 || s.dilation != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
     if (c.NT != 1 || c.need_xchg || c.padded || c.nacc != 2) return false;
     if (c.d2_col + C2 > c.tmem_cols) return false;

@@ -122,6 +122,42 @@ def test_copy_warp_producer_shapes(cfg):
     check_layer(L, seed=23)
 
 
+# Dilated 3x3 (pad = dilation) on the tensor-core variant: vertical taps become shifts by `dilation` rows, horizontal
+# ones lane shifts by `dilation` columns inside a 32-pixel segment, so only planes whose rows divide 32 pixels
+# (after padding the width to a multiple of 4) are taken: 32, 16 and 8 wide, 14 (copy warps) and 7.
+DILATED_SHAPES = [
+    (2, 32, 32, 32, 32, 3, 3, 1, 2, 2, 4), (3, 64, 16, 16, 64, 3, 3, 1, 2, 2, 2), (4, 128, 8, 8, 128, 3, 3, 1, 3, 3, 8),
+    (5, 32, 14, 14, 32, 3, 3, 1, 2, 2, 4), (2, 64, 16, 16, 128, 3, 3, 1, 4, 4, 1), (2, 32, 7, 7, 32, 3, 3, 1, 2, 2, 1),
+    (1, 16, 32, 32, 16, 3, 3, 1, 5, 5, 2), (130, 64, 32, 32, 64, 3, 3, 1, 2, 2, 8), (9, 32, 24, 16, 48, 3, 3, 1, 6, 6, 1),
+    (3, 256, 14, 14, 256, 3, 3, 1, 2, 2, 1), (2, 16, 40, 8, 16, 3, 3, 1, 9, 9, 2),
+]
+
+
+@pytest.mark.parametrize("cfg", DILATED_SHAPES)
+def test_dilated_shapes_on_the_tensor_core_variant(cfg):
+    L = Layer("dilated", *cfg)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32
+    finally:
+        gconv.gconv_desc_destroy(d)
+    check_layer(L, seed=29)
+    check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=29)
+
+
+def test_dilation_the_tensor_core_variant_does_not_take():
+    """Rows that do not divide a segment, pad != dilation, stride 2: the selector falls back and the result still agrees."""
+    for cfg in ((1, 16, 28, 28, 16, 3, 3, 1, 2, 2, 2), (1, 16, 16, 16, 16, 3, 3, 1, 1, 2, 2), (1, 16, 16, 16, 16, 3, 3, 2, 2, 2, 2)):
+        L = Layer("dilated_fallback", *cfg)
+        d = gconv.gconv_desc_create(*L.desc_args())
+        try:
+            assert gconv.gconv_variant(d) != gconv.GCONV_VARIANT_IGEMM_TF32
+            assert not gconv.gconv_variant_supported(d, gconv.GCONV_VARIANT_IGEMM_TF32)
+        finally:
+            gconv.gconv_desc_destroy(d)
+        check_layer(L, seed=30)
+
+
 @pytest.mark.parametrize("groups", [1, 2, 4, 8, 16])
 def test_wrn_stack_small_batch(groups):
     """Every distinct layer of the WRN-40-2-shaped stack at N = 1 and a ragged N = 3, all variants."""
