@@ -419,15 +419,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2 instead
         // of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
         // Pass 1 is the real one.
-        for (int pass = (c.soft ? 1 : 0); pass < 2 && ok; ++pass) {
-        const bool pf = pass == 0;
-        if (!pf) {
-            asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
-            it = 0;
-            stage = 0;
-            ph = 0;
-        }
-        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile = tile_next(tile)) {
+        // One tile's stages: the real copies (arming the stage barriers), or -- pf -- only L2 prefetches of the first
+        // pf_limit of them (no barrier).  (Asking L2 for the CTA's next tile while the current one is in flight was
+        // measured too: 2 % slower on the stack.)
+        auto visit = [&](const int tile, const bool pf, const uint32_t pf_limit, uint32_t& it, int& stage, uint32_t& ph) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
             uint32_t gq = gn, ntq = 0;
@@ -439,7 +434,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 // the copy warps stage the input; this warp only brings the resident weights of a new (group, filter tile)
                 if (switch_b) {
                     const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
-                    if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; break; }
+                    if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; return; }
                     const uint32_t bar = smem_u32(&ctl.b_full[bb]);
                     if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
                     __syncwarp();
@@ -448,7 +443,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     cur_gn = (int)gn;
                     ++switches;
                 }
-                continue;
+                return;
             }
             // Whole-tile copies: a row-box tile is always one 5-D box; a flat tile whose segments are one contiguous run
             // is one 4-D box for every tap whose run stays inside the image plane.  Everything else (tiles that straddle
@@ -471,7 +466,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             bool have_lane_coords = false;
             int ch = 0, r = c.nr == 3 ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
-                if (pf && it >= kPrefetchUses) break;
+                if (pf && it >= pf_limit) break;
                 // the first pass over the ring finds every stage free
                 if (!pf && it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
@@ -539,6 +534,17 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
+        };
+        for (int pass = (c.soft ? 1 : 0); pass < 2 && ok; ++pass) {
+        const bool pf = pass == 0;
+        if (!pf) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
+            it = 0;
+            stage = 0;
+            ph = 0;
+        }
+        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile = tile_next(tile)) {
+            visit(tile, pf, kPrefetchUses, it, stage, ph);
         }
         }
         if (!ok && lane == 0) {
