@@ -53,11 +53,9 @@ __device__ __forceinline__ void strow(float* __restrict__ dst, int col, int W, c
 }
 
 // ---- stride 1 -------------------------------------------------------------------------------------
-__device__ __forceinline__ void row_taps1(const float4 v, bool has_l, bool has_r, const float (&w)[3], float (&acc)[4]) {
-    float l = __shfl_up_sync(0xffffffffu, v.w, 1);
-    float r = __shfl_down_sync(0xffffffffu, v.x, 1);
-    l = has_l ? l : 0.f;
-    r = has_r ? r : 0.f;
+// One input row's contribution to an output row: v = the strip's own four columns, l / r = the columns just left and
+// right of it (from the neighbouring lanes, zero at the image border).
+__device__ __forceinline__ void row_taps1(const float4 v, const float l, const float r, const float (&w)[3], float (&acc)[4]) {
     acc[0] = fmaf(l, w[0], acc[0]);   acc[0] = fmaf(v.x, w[1], acc[0]); acc[0] = fmaf(v.y, w[2], acc[0]);
     acc[1] = fmaf(v.x, w[0], acc[1]); acc[1] = fmaf(v.y, w[1], acc[1]); acc[1] = fmaf(v.z, w[2], acc[1]);
     acc[2] = fmaf(v.y, w[0], acc[2]); acc[2] = fmaf(v.z, w[1], acc[2]); acc[2] = fmaf(v.w, w[2], acc[2]);
@@ -65,7 +63,7 @@ __device__ __forceinline__ void row_taps1(const float4 v, bool has_l, bool has_r
 }
 
 template <int VEC>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, VEC == 0 ? 2 : 3)   // three blocks per SM (80 registers) unless the scalar loads would spill
 dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
     const uint32_t tag_seen = __ldg(packed);
@@ -90,10 +88,20 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
 #pragma unroll
     for (int i = 0; i < 9; ++i) w[i / 3][i % 3] = live ? __ldg(wpk + (size_t)ch * 9 + i) : 0.f;
 
-    // rows p-1 .. p+U of the current block; `live` only gates memory traffic, every lane runs the shuffles
+    // rows p-1 .. p+U of the current block; `live` only gates memory traffic, every lane runs the shuffles.  A row
+    // feeds three output rows, so its two halo columns are fetched from the neighbouring lanes once, when the row
+    // enters the block, and kept (hl, hr).
     float4 cur[U + 2], nxt[U];
+    float hl[U + 2], hr[U + 2];
+    auto halo = [&](const float4 v, float& l, float& r) {
+        const float a = __shfl_up_sync(0xffffffffu, v.w, 1), b = __shfl_down_sync(0xffffffffu, v.x, 1);
+        l = has_l ? a : 0.f;
+        r = has_r ? b : 0.f;
+    };
 #pragma unroll
     for (int j = 0; j < U + 2; ++j) cur[j] = live ? ldrow<VEC>(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < U + 2; ++j) halo(cur[j], hl[j], hr[j]);
     for (int p = p0; p < p0 + c.RH; p += U) {        // warp-uniform trip count
 #pragma unroll
         for (int j = 0; j < U; ++j) {                  // next block's new rows, in flight during this block's math
@@ -103,15 +111,20 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            row_taps1(cur[j], has_l, has_r, w[0], acc);
-            row_taps1(cur[j + 1], has_l, has_r, w[1], acc);
-            row_taps1(cur[j + 2], has_l, has_r, w[2], acc);
+            row_taps1(cur[j], hl[j], hr[j], w[0], acc);
+            row_taps1(cur[j + 1], hl[j + 1], hr[j + 1], w[1], acc);
+            row_taps1(cur[j + 2], hl[j + 2], hr[j + 2], w[2], acc);
             if (live && p + j < p1 && tag_seen == tag) strow<VEC>(yp + (size_t)(p + j) * s.W + col, col, s.W, acc);
         }
         cur[0] = cur[U];
         cur[1] = cur[U + 1];
+        hl[0] = hl[U]; hr[0] = hr[U];
+        hl[1] = hl[U + 1]; hr[1] = hr[U + 1];
 #pragma unroll
-        for (int j = 0; j < U; ++j) cur[2 + j] = nxt[j];
+        for (int j = 0; j < U; ++j) {
+            cur[2 + j] = nxt[j];
+            halo(nxt[j], hl[2 + j], hr[2 + j]);
+        }
     }
     if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 }
