@@ -411,7 +411,15 @@ DwCfg dw_config(const Shape& s, int sm_count) {
     const long long planes = (long long)s.N * s.C_in;
     const long long want = s.KH == 5 ? 410LL * sm_count : 6LL * 1024 * sm_count;
     int rh = s.H_out;
-    while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < want) rh = (rh + 1) / 2;
+    if (s.KH == 3 && s.stride == 1 && s.H_out >= 28) {
+        // 3x3 stride 1 on planes of 28 rows and more: strips of 28 rows measured best at 28x28, 56x56 and 112x112
+        // (7 % halo rows, long enough to amortise the set-up) as long as about half a wave of lanes remains
+        rh = 28;
+        while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < 512LL * sm_count) rh = (rh + 1) / 2;
+    } else {
+        while (rh > 8 && planes * ((s.H_out + rh - 1) / rh) * c.XQ < want) rh = (rh + 1) / 2;
+        if (s.KH == 3 && s.stride == 1 && s.H_out <= 8 && planes * c.XQ * 2 >= 512LL * sm_count) rh = 4;   // 7x7, 8x8: two short strips
+    }
     rh = ((rh + U - 1) / U) * U;
     c.RH = rh;
     c.chunks = (s.H_out + rh - 1) / rh;
