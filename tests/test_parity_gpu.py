@@ -122,6 +122,20 @@ def test_copy_warp_producer_shapes(cfg):
     check_layer(L, seed=23)
 
 
+# Two filter tiles per group (80 filters: two tiles of 40) in the two-CTA launch shape, alone and with several groups,
+# on segment tilings, row boxes and stride-2 row tiles.
+TWO_FILTER_TILE_SHAPES = [
+    (4, 16, 16, 16, 80, 3, 3, 1, 1, 1, 1), (40, 32, 16, 16, 160, 3, 3, 1, 1, 1, 2), (3, 16, 32, 32, 80, 3, 3, 1, 1, 1, 1),
+    (130, 16, 8, 8, 80, 3, 3, 1, 1, 1, 1), (5, 16, 28, 28, 80, 3, 3, 1, 1, 1, 1), (6, 16, 32, 32, 80, 3, 3, 2, 1, 1, 1),
+    (128, 64, 16, 16, 320, 3, 3, 2, 1, 1, 4),
+]
+
+
+@pytest.mark.parametrize("cfg", TWO_FILTER_TILE_SHAPES)
+def test_two_filter_tiles_per_group(cfg):
+    check_layer(Layer("nt2", *cfg), seed=37)
+
+
 # Dilated 3x3 (pad = dilation) on the tensor-core variant: vertical taps become shifts by `dilation` rows, horizontal
 # ones lane shifts by `dilation` columns inside a 32-pixel segment, so only planes whose rows divide 32 pixels
 # (after padding the width to a multiple of 4) are taken: 32, 16 and 8 wide, 14 (copy warps) and 7.
