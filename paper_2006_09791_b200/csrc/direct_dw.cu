@@ -131,9 +131,8 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
 
 // ---- stride 2 -------------------------------------------------------------------------------------
 // Four outputs q..q+3 read input columns 2q-1 .. 2q+7: two aligned float4 (a, b) and the previous lane's b.w.
-__device__ __forceinline__ void row_taps2(const float4 a, const float4 b, bool has_l, const float (&w)[3], float (&acc)[4]) {
-    float l = __shfl_up_sync(0xffffffffu, b.w, 1);
-    l = has_l ? l : 0.f;
+// (l = the column just left of the strip: the previous lane's b.w, zero at the image border)
+__device__ __forceinline__ void row_taps2(const float4 a, const float4 b, const float l, const float (&w)[3], float (&acc)[4]) {
     acc[0] = fmaf(l, w[0], acc[0]);   acc[0] = fmaf(a.x, w[1], acc[0]); acc[0] = fmaf(a.y, w[2], acc[0]);
     acc[1] = fmaf(a.y, w[0], acc[1]); acc[1] = fmaf(a.z, w[1], acc[1]); acc[1] = fmaf(a.w, w[2], acc[1]);
     acc[2] = fmaf(a.w, w[0], acc[2]); acc[2] = fmaf(b.x, w[1], acc[2]); acc[2] = fmaf(b.y, w[2], acc[2]);
@@ -175,6 +174,9 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
         ca[j] = live ? ldrow<VEC>(xp, 2 * p0 + j, s.H, s.W, col) : z4;
         cb[j] = (live && second_ok) ? ldrow<VEC>(xp, 2 * p0 + j, s.H, s.W, col + 4) : z4;
     }
+    // the left halo of a row is fetched from the neighbouring lane once; the bottom row of one output is the top row of the next
+    auto halo = [&](const float4 b) { const float v = __shfl_up_sync(0xffffffffu, b.w, 1); return has_l ? v : 0.f; };
+    float lt = halo(tb), lc[2] = {halo(cb[0]), halo(cb[1])};
     for (int p = p0; p < p0 + c.RH; ++p) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {                  // rows of the next output, in flight during this one's math
@@ -184,9 +186,9 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
             nb[j] = (need && second_ok) ? ldrow<VEC>(xp, h, s.H, s.W, col + 4) : z4;
         }
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        row_taps2(ta, tb, has_l, w[0], acc);
-        row_taps2(ca[0], cb[0], has_l, w[1], acc);
-        row_taps2(ca[1], cb[1], has_l, w[2], acc);
+        row_taps2(ta, tb, lt, w[0], acc);
+        row_taps2(ca[0], cb[0], lc[0], w[1], acc);
+        row_taps2(ca[1], cb[1], lc[1], w[2], acc);
         if (live && p < p1 && tag_seen == tag) {
             float* dst = yp + (size_t)p * s.W_out + xq * 4;
             if ((s.W_out & 3) == 0) {
@@ -202,8 +204,9 @@ dw_stream_s2_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
         }
         ta = ca[1];
         tb = cb[1];
+        lt = lc[1];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) { ca[j] = na[j]; cb[j] = nb[j]; }
+        for (int j = 0; j < 2; ++j) { ca[j] = na[j]; cb[j] = nb[j]; lc[j] = halo(nb[j]); }
     }
     if (tag_seen != tag && threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
 }
