@@ -14,7 +14,7 @@ namespace gconv {
 
 namespace {
 
-constexpr int U = 4;   // output rows per pipeline block
+constexpr int U = 4;   // output rows per pipeline block (strip lengths are multiples of it)
 
 // Four consecutive pixels of row h starting at column col (zero outside the image).  VEC = 4: W % 4 == 0, so the
 // address is 16-byte aligned and the four pixels are in range; VEC = 2: W is even, two 8-byte loads (the second pair
@@ -62,8 +62,10 @@ __device__ __forceinline__ void row_taps1(const float4 v, const float l, const f
     acc[3] = fmaf(v.z, w[0], acc[3]); acc[3] = fmaf(v.w, w[1], acc[3]); acc[3] = fmaf(r, w[2], acc[3]);
 }
 
-template <int VEC>
-__global__ void __launch_bounds__(256, VEC == 0 ? 2 : 3)   // three blocks per SM (80 registers) unless the scalar loads would spill
+// UB = output rows per pipeline block: 4 on planes of 28 rows and more (80 registers, three blocks per SM), 2 on smaller
+// ones (64 registers, four blocks per SM: short strips want more warps rather than more rows in flight per thread).
+template <int VEC, int UB>
+__global__ void __launch_bounds__(256, VEC == 0 ? 2 : (UB == 4 ? 3 : 4))
 dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                     float* __restrict__ y, Status* status, uint32_t tag) {
     const uint32_t tag_seen = __ldg(packed);
@@ -88,40 +90,40 @@ dw_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, c
 #pragma unroll
     for (int i = 0; i < 9; ++i) w[i / 3][i % 3] = live ? __ldg(wpk + (size_t)ch * 9 + i) : 0.f;
 
-    // rows p-1 .. p+U of the current block; `live` only gates memory traffic, every lane runs the shuffles.  A row
+    // rows p-1 .. p+UB of the current block; `live` only gates memory traffic, every lane runs the shuffles.  A row
     // feeds three output rows, so its two halo columns are fetched from the neighbouring lanes once, when the row
     // enters the block, and kept (hl, hr).
-    float4 cur[U + 2], nxt[U];
-    float hl[U + 2], hr[U + 2];
+    float4 cur[UB + 2], nxt[UB];
+    float hl[UB + 2], hr[UB + 2];
     auto halo = [&](const float4 v, float& l, float& r) {
         const float a = __shfl_up_sync(0xffffffffu, v.w, 1), b = __shfl_down_sync(0xffffffffu, v.x, 1);
         l = has_l ? a : 0.f;
         r = has_r ? b : 0.f;
     };
 #pragma unroll
-    for (int j = 0; j < U + 2; ++j) cur[j] = live ? ldrow<VEC>(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < UB + 2; ++j) cur[j] = live ? ldrow<VEC>(xp, p0 - 1 + j, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < U + 2; ++j) halo(cur[j], hl[j], hr[j]);
-    for (int p = p0; p < p0 + c.RH; p += U) {        // warp-uniform trip count
+    for (int j = 0; j < UB + 2; ++j) halo(cur[j], hl[j], hr[j]);
+    for (int p = p0; p < p0 + c.RH; p += UB) {        // warp-uniform trip count
 #pragma unroll
-        for (int j = 0; j < U; ++j) {                  // next block's new rows, in flight during this block's math
-            const int h = p + U + 1 + j;
+        for (int j = 0; j < UB; ++j) {                  // next block's new rows, in flight during this block's math
+            const int h = p + UB + 1 + j;
             nxt[j] = (live && h <= p1) ? ldrow<VEC>(xp, h, s.H, s.W, col) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int j = 0; j < U; ++j) {
+        for (int j = 0; j < UB; ++j) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
             row_taps1(cur[j], hl[j], hr[j], w[0], acc);
             row_taps1(cur[j + 1], hl[j + 1], hr[j + 1], w[1], acc);
             row_taps1(cur[j + 2], hl[j + 2], hr[j + 2], w[2], acc);
             if (live && p + j < p1 && tag_seen == tag) strow<VEC>(yp + (size_t)(p + j) * s.W + col, col, s.W, acc);
         }
-        cur[0] = cur[U];
-        cur[1] = cur[U + 1];
-        hl[0] = hl[U]; hr[0] = hr[U];
-        hl[1] = hl[U + 1]; hr[1] = hr[U + 1];
+        cur[0] = cur[UB];
+        cur[1] = cur[UB + 1];
+        hl[0] = hl[UB]; hr[0] = hr[UB];
+        hl[1] = hl[UB + 1]; hr[1] = hr[UB + 1];
 #pragma unroll
-        for (int j = 0; j < U; ++j) {
+        for (int j = 0; j < UB; ++j) {
             cur[2 + j] = nxt[j];
             halo(nxt[j], hl[2 + j], hr[2 + j]);
         }
@@ -445,7 +447,11 @@ cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float
     } while (0)
 #define GCONV_DW5_S1(V) dw5_stream_s1_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
 #define GCONV_DW5_S2(V) dw5_stream_kernel<V, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
-#define GCONV_DW3_S1(V) dw_stream_s1_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
+#define GCONV_DW3_S1(V) \
+    do { \
+        if (s.H_out >= 28) dw_stream_s1_kernel<V, 4><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag); \
+        else dw_stream_s1_kernel<V, 2><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag); \
+    } while (0)
 #define GCONV_DW3_S2(V) dw_stream_s2_kernel<V><<<c.blocks, 256, 0, st>>>(s, c, x, pk, y, status, tag)
     if (s.KH == 5) {
         if (s.stride == 1) GCONV_DW_LAUNCH(GCONV_DW5_S1);
