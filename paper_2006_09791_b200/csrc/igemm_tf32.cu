@@ -652,15 +652,18 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 }
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const float* xg = x + ((size_t)(img_ok ? n : 0u) * s.C_in + (size_t)((int)gq * c.Cg + ch * c.CK)) * plane;
-                const int ntb = c.tapb ? 3 : 1;
-                for (int tb = 0; tb < ntb; ++tb) {
-                    const int tap = c.tapb ? tb : r;
-                    const int f = (int)i * c.seg_fstep + (tap - 1) * rstep + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
+                // this warp's 32-pixel blocks of the stage: block pw, pw + 4, ...  A halo stage (rows of one segment) holds
+                // the tile's rows and the rows above and below, block b = padded row b - wseg of the tile; a tap-block
+                // stage holds three shifted copies of the tile, block 4 * tap + segment; else one block per segment
+                const bool halo = c.nr == 3 && !c.tapb;
+                for (int b = pw, kb = 0; b < c.nseg; b += kSoftWarps, ++kb) {
+                    const int f0 = halo ? ((int)i + 4 * kb - c.wseg) * 32 : (int)i * c.seg_fstep + ((c.tapb ? kb : r) - 1) * rstep;
+                    const int f = f0 + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
                     const int row = f >> wshift, col = f & (s.W - 1);
                     const bool valid = img_ok && f >= 0 && row < c.Hv && col < c.Wv;
                     const float* src = valid ? xg + (size_t)row * c.Wv + col : x;
                     const uint32_t nbytes = valid ? (pairs ? 8u : 4u) : 0u;
-                    const uint32_t dseg = a_dst + (uint32_t)(tb * 4 + pw) * seg_bytes + unit_in;
+                    const uint32_t dseg = a_dst + (uint32_t)b * seg_bytes + unit_in;
                     if (pairs) {
                         for (int k = kfirst; k < c.CK; k += kstep)
                             asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dseg + (uint32_t)k * 128u + ((unit_chunk ^ ((uint32_t)k & 3u)) << 5)),

@@ -107,6 +107,7 @@ COPY_WARP_SHAPES = [
     (3, 24, 10, 6, 24, 3, 3, 1, 1, 1, 3), (4, 32, 15, 15, 32, 3, 3, 1, 1, 1, 1), (2, 8, 9, 31, 16, 3, 3, 1, 1, 1, 1),
     (7, 32, 7, 7, 32, 3, 3, 2, 1, 1, 4), (300, 64, 14, 14, 64, 3, 3, 1, 1, 1, 2), (40, 512, 14, 14, 512, 3, 3, 1, 1, 1, 32),
     (33, 256, 7, 7, 256, 3, 3, 1, 1, 1, 8), (1, 8, 5, 7, 8, 3, 3, 1, 1, 1, 1), (6, 48, 13, 14, 96, 3, 3, 1, 1, 1, 6),
+    (3, 512, 56, 30, 512, 3, 3, 1, 1, 1, 64), (5, 32, 28, 31, 32, 3, 3, 1, 1, 1, 2), (2, 16, 8, 29, 16, 3, 3, 1, 1, 1, 1),   # halo stages
 ]
 
 
