@@ -207,9 +207,9 @@ def test_mobilenetv2_depthwise_shapes():
 
 
 def _seeded_random_shapes(seed, count):
-    """3x3, pad 1 layers drawn from the sizes the selector, the tilings and the kernel families branch on (plane
-    sizes around the 32-pixel segment and the 128-pixel tile, widths that need padding, narrow and wide groups,
-    unequal Cg and Kg, both strides, ragged batches), each small enough for the oracle."""
+    """3x3, pad = dilation layers drawn from the sizes the selector, the tilings and the kernel families branch on (plane
+    sizes around the 32-pixel segment and the 128-pixel tile, widths that need padding or copy warps, narrow and wide
+    groups, unequal Cg and Kg, both strides, dilation 1 to 3, ragged batches), each small enough for the oracle."""
     import random
     rng = random.Random(seed)
     out = []
@@ -220,18 +220,21 @@ def _seeded_random_shapes(seed, count):
         C, K = g * cg, g * kg
         if C > 512 or K > 512:
             continue
-        H = rng.choice([7, 8, 9, 14, 15, 16, 17, 27, 28, 30, 31, 32, 33, 40, 55, 56, 57, 64])
-        W = rng.choice([7, 8, 12, 14, 16, 20, 24, 28, 30, 32, 36, 40, 48, 52, 56, 60, 64, 96, 128])
+        H = rng.choice([5, 7, 8, 9, 14, 15, 16, 17, 27, 28, 30, 31, 32, 33, 40, 55, 56, 57, 64])
+        W = rng.choice([5, 6, 7, 8, 12, 13, 14, 15, 16, 20, 24, 28, 29, 30, 31, 32, 36, 40, 48, 52, 56, 60, 64, 96, 128])
         stride = rng.choice([1, 1, 1, 2])
+        dil = rng.choice([1, 1, 1, 1, 2, 3])
+        if H <= 2 * dil or W <= 2 * dil:
+            dil = 1
         macs_per_image = C // g * K * 9 * ((H - 1) // stride + 1) * ((W - 1) // stride + 1)
         N = min(rng.choice([1, 2, 3, 5, 8, 13, 32, 64, 128, 200]), max(1, int(1.5e9 // macs_per_image)))
         if N * C * H * W > 40e6:
             continue
-        out.append((N, C, H, W, K, 3, 3, stride, 1, 1, g))
+        out.append((N, C, H, W, K, 3, 3, stride, dil, dil, g))
     return out
 
 
-@pytest.mark.parametrize("chunk", range(4))
+@pytest.mark.parametrize("chunk", range(6))
 def test_seeded_random_shapes(chunk):
     for i, cfg in enumerate(_seeded_random_shapes(20260 + chunk, 25)):
         check_layer(Layer("rand%d_%d" % (chunk, i), *cfg), seed=100 * chunk + i)
