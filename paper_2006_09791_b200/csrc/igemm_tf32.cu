@@ -1029,7 +1029,9 @@ __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__
             const int gi = ke / s.Kg;                        // which original group of the merge
             if (ce / s.Cg == gi) {
                 const int ko = (g * c.merge + gi) * s.Kg + (ke - gi * s.Kg);
-                const float v = w[(((size_t)ko) * s.Cg + (ce - gi * s.Cg)) * 9 + r * 3 + ss];
+                // a pointwise (1x1) filter is the centre tap of a 3x3 filter whose other taps are zero
+                const size_t wi = ((size_t)ko) * s.Cg + (ce - gi * s.Cg);
+                const float v = s.KH == 1 ? ((r == 1 && ss == 1) ? w[wi] : 0.f) : w[wi * 9 + r * 3 + ss];
                 asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(bits) : "f"(v));
             }
         }
@@ -1063,6 +1065,19 @@ struct IgemmGeom {
     int Hp, Wp;
     bool padded;
 };
+// A pointwise convolution (1x1, pad 0) runs as the 3x3, pad 1 convolution whose only non-zero tap is the centre one
+// (same output size for either stride); the packing kernel writes the zeros.
+static Shape as_3x3(const Shape& s) {
+    Shape t = s;
+    if (s.KH == 1 && s.KW == 1) {
+        t.KH = 3;
+        t.KW = 3;
+        t.pad = 1;
+        t.dilation = 1;
+    }
+    return t;
+}
+
 static IgemmGeom igemm_geom(const Shape& s) {
     IgemmGeom g;
     g.Wp = (s.W + 3) & ~3;
@@ -1121,7 +1136,9 @@ static int igemm_merge(const Shape& s) {
     return m;
 }
 
-bool igemm_supported(const Shape& s) {
+bool igemm_supported(const Shape& s_any) {
+    if (s_any.KH == 1 && s_any.KW == 1 && !(s_any.pad == 0 && s_any.dilation == 1)) return false;
+    const Shape s = as_3x3(s_any);
     if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.dilation >= 1 && s.pad == s.dilation)) return false;
     if (s.dilation > 1 && (s.stride != 1 || s.dilation > 16)) return false;
     const int m = igemm_merge(s);
@@ -1143,7 +1160,8 @@ size_t igemm_scratch_bytes(const Shape& s) {
     return sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp;
 }
 
-static IgemmCfg igemm_config_c2(const Shape& s_true, int sm_count, int C2) {
+static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
+    const Shape s_true = as_3x3(s_any);
     IgemmCfg c;
     const bool fuse = C2 > 0;          // fused grouped + pointwise block: heavy shape, streamed or resident grouped weights
     const IgemmGeom ge = igemm_geom(s_true);
@@ -1367,7 +1385,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, 
 
 // ---- fused block: grouped 3x3 followed by a pointwise (1x1, groups = 1) convolution C_out -> C2 ------------------------
 bool igemm_block_supported(const Shape& s, int C2) {
-    if (!igemm_supported(s) || s.stride != 1 || s.dilation != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
+    if (!igemm_supported(s) || s.KH != 3 || s.stride != 1 || s.dilation != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
     if (c.NT != 1 || c.need_xchg || c.padded || c.nacc != 2) return false;
     if (c.d2_col + C2 > c.tmem_cols) return false;
@@ -1445,7 +1463,7 @@ cudaError_t igemm_block_forward(const Shape& s, int C2, const float* x, const vo
 static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, const void* packed, float* y, Status* status,
                                 int sm_count, cudaStream_t st, float* scratch) {
     const IgemmCfg c = igemm_config_c2(s_true, sm_count, C2);
-    Shape s = s_true;
+    Shape s = as_3x3(s_true);
     const float* x = x_in;
     if (c.padded) {
         if (scratch == nullptr) return cudaErrorInvalidValue;

@@ -137,6 +137,26 @@ def test_two_filter_tiles_per_group(cfg):
     check_layer(Layer("nt2", *cfg), seed=37)
 
 
+# Pointwise (1x1, pad 0) convolutions: the tensor-core variant runs them as the centre tap of a 3x3 filter.
+POINTWISE_SHAPES = [
+    (8, 64, 16, 16, 64, 1, 1, 1, 0, 1, 1), (3, 32, 32, 32, 128, 1, 1, 1, 0, 1, 1), (5, 256, 14, 14, 256, 1, 1, 1, 0, 1, 1),
+    (4, 64, 16, 16, 128, 1, 1, 2, 0, 1, 1), (2, 256, 28, 28, 256, 1, 1, 1, 0, 1, 1), (130, 32, 32, 32, 32, 1, 1, 1, 0, 1, 4),
+    (7, 128, 7, 7, 64, 1, 1, 1, 0, 1, 2), (2, 64, 56, 56, 256, 1, 1, 1, 0, 1, 1), (3, 48, 20, 24, 96, 1, 1, 2, 0, 1, 3),
+]
+
+
+@pytest.mark.parametrize("cfg", POINTWISE_SHAPES)
+def test_pointwise_on_the_tensor_core_variant(cfg):
+    L = Layer("pointwise", *cfg)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32
+    finally:
+        gconv.gconv_desc_destroy(d)
+    check_layer(L, seed=41)
+    check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=41)
+
+
 # Dilated 3x3 (pad = dilation) on the tensor-core variant: vertical taps become shifts by `dilation` rows, horizontal
 # ones lane shifts by `dilation` columns inside a 32-pixel segment, so only planes whose rows divide 32 pixels
 # (after padding the width to a multiple of 4) are taken: 32, 16 and 8 wide, 14 (copy warps) and 7.
