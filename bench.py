@@ -275,9 +275,10 @@ def time_block(torch, gconv, L, C2, stream, reps=20, min_cycle_bytes=2 * L2_BYTE
         gconv.gconv_desc_destroy(d)
 
 
-def block_row(L, C2, ms_block, ms_grouped, peaks):
-    """Fused grouped + pointwise block: its time against the HBM floor of the block (x in, y2 out) and against the
-    unfused pair's floor (the grouped layer as measured alone, plus reading y1 and writing y2 at the HBM peak)."""
+def block_row(L, C2, ms_block, ms_grouped, ms_pointwise, peaks):
+    """Fused grouped + pointwise block: its time against the HBM floor of the block (x in, y2 out), against the
+    unfused pair as measured (the grouped layer and the pointwise layer, each timed alone through gconv_forward) and
+    against that pair's floor (the grouped layer as measured, plus reading y1 and writing y2 at the HBM peak)."""
     hbm = peaks["hbm_gbs"] * 1e9
     pix = L.N * L.H_out * L.W_out
     bytes_block = 4 * (L.x_elems + pix * C2)
@@ -286,6 +287,7 @@ def block_row(L, C2, ms_block, ms_grouped, peaks):
     t_roof = max(bytes_block / hbm, t_tensor)
     unfused_floor_ms = ms_grouped + 4e3 * pix * (L.C_out + C2) / hbm
     return {"layer": L.name, "groups": L.groups, "N": L.N, "C2": C2, "ms": ms_block, "grouped_only_ms": ms_grouped,
+            "pointwise_only_ms": ms_pointwise, "unfused_measured_ms": ms_grouped + ms_pointwise,
             "unfused_floor_ms": unfused_floor_ms, "gflops": flops / (ms_block * 1e-3) / 1e9,
             "gbs": bytes_block / (ms_block * 1e-3) / 1e9, "roofline_ms": t_roof * 1e3,
             "bound": "hbm" if bytes_block / hbm >= t_tensor else "tensor", "roofline_frac": t_roof / (ms_block * 1e-3)}
@@ -523,7 +525,9 @@ def run_ours(args):
                 msb = time_block(torch, gconv, L, C2, stream)
                 if msb is not None:
                     msg, _ = time_layer(torch, gconv, L, stream, reps=20)
-                    block_rows.append(block_row(L, C2, msb, msg, peaks))
+                    Lp = wl.Layer(L.name + "_pw", L.N, L.C_out, L.H_out, L.W_out, C2, 1, 1, 1, 0, 1, 1)
+                    msp, _ = time_layer(torch, gconv, Lp, stream, reps=20)
+                    block_rows.append(block_row(L, C2, msb, msg, msp, peaks))
             extra["fused_blocks"] = block_rows
             extra["stack_n1_chained_ms_by_groups"] = {str(g): chained_stack_ms(torch, gconv, g, stream) for g in wl.WRN_GROUPS}
 

@@ -58,8 +58,9 @@ enum gconv_variant_id {
     GCONV_VARIANT_DIRECT_GENERIC = 1, /* FP32 FFMA, one thread per output, any shape */
     GCONV_VARIANT_DIRECT_TILED = 2,   /* FP32 FFMA, shared-memory halo + register tiles; 3x3, dilation 1, narrow groups;
                                          depthwise 3x3 (pad 1) and 5x5 (pad 2) on a software-pipelined stream kernel */
-    GCONV_VARIANT_IGEMM_TF32 = 3      /* TF32 tcgen05 implicit GEMM per (merged) group; 3x3, pad = dilation, stride 1 or 2, W <= 128;
-                                         dilation > 1 only with stride 1 on planes whose (padded) rows divide 32 pixels */
+    GCONV_VARIANT_IGEMM_TF32 = 3      /* TF32 tcgen05 implicit GEMM per (merged) group; 3x3 with pad = dilation or 1x1 with pad 0,
+                                         stride 1 or 2, W <= 128; dilation > 1 only with stride 1 on planes whose (padded)
+                                         rows divide 32 pixels */
 };
 
 /*

@@ -126,6 +126,7 @@ struct IgemmCfg {
     int tapb;                // one stage holds three blocks of four segments, one per vertical tap (small planes)
     // fused grouped + pointwise block (0 for the plain convolution)
     int fuse, C2, n_gn, d2_col;   // pointwise output channels, (group, filter tile) pairs per pixel tile, TMEM column of its accumulator
+    int pw;                       // pointwise layer, stride 1: one vertical tap per chunk, one accumulator per filter (N = Kt)
     int soft;                     // copy warps stage the input with cp.async (widths TMA cannot address); no padded copy of x
     int ball;                     // every (group, filter tile) keeps a resident weight buffer of its own: no switches
     int d2_bufs;                  // pointwise accumulators in TMEM (2 when the columns allow: alternate pixel tiles)

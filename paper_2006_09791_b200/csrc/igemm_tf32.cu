@@ -230,32 +230,34 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft;
+        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw;
 };
-constexpr int kFamilies = 17;
+constexpr int kFamilies = 19;
 __host__ __device__ constexpr Family family(int f) {
-    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft
-    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
-         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0,  0}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0,  0}     // row boxes of two segments, narrow groups
-         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
-         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0}     // stride-2 row tiles, narrow groups
-         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
-         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
-         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0,  0}     // row boxes of one segment, narrow groups
-         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
-         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0}     // fused block, 32-wide planes with halo stages
-         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1,  0}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
-         : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0}     // fused block, 32-wide planes, two CTAs per SM
-         : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0}     // fused block, row boxes, two resident banks
-         : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1}     // copy-warp producer (14x14, 7x7 planes), tap blocks
-         : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1}     // copy-warp producer, one stage per tap
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1};
+    //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
+    return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
+         : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0,  0,  0}     // 32-wide planes with halo stages
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0,  0,  0}     // row boxes of two segments, narrow groups
+         : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
+         : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, narrow groups
+         : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
+         : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
+         : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0,  0,  0}     // row boxes of one segment, narrow groups
+         : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
+         : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0,  0}     // fused block, 32-wide planes with halo stages
+         : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1,  0,  0}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
+         : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0,  0}     // fused block, 32-wide planes, two CTAs per SM
+         : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0,  0}     // fused block, row boxes, two resident banks
+         : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1,  0}     // copy-warp producer (14x14, 7x7 planes), tap blocks
+         : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1,  0}     // copy-warp producer, one stage per tap
+         : f == 17 ? Family{0,  1,  1,  0,   1,  1,  0,  1,  1, 32, -1, -1,  -1,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, two CTAs per SM
+         : f == 18 ? Family{1,  0,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0, -1,  0,   4, -1,  1,  0,  0,  0,  0,  1}     // pointwise, row boxes
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball) X(soft)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball) X(soft) X(pw)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -354,11 +356,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     // Pipeline geometry.  A stage holds the input segments of one channel chunk: either the four
     // segments of one vertical tap (nr = 1, stages run chunk-major, tap-minor), or the tile plus its
     // row halo (nr = 3: the three taps are views of the same stage, shifted by whole segments).
-    const int kstages = (3 / c.nr) * c.chunks;
+    const int vt = c.pw ? 1 : 3;                 // vertical taps (a pointwise layer has one tap, no neighbours)
+    const int kstages = (vt / c.nr) * c.chunks;
     const uint32_t seg_bytes = (uint32_t)c.CK * 128u;
     const uint32_t a_bytes = (uint32_t)c.nseg * seg_bytes;
     const uint32_t blk_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;   // weights of one (chunk, tap)
-    const uint32_t b_tile_bytes = 3u * (uint32_t)c.chunks * blk_bytes;   // weights of one (group, filter tile)
+    const uint32_t b_tile_bytes = (uint32_t)vt * (uint32_t)c.chunks * blk_bytes;   // weights of one (group, filter tile)
     const uint32_t bres_base = smem_base;                                // two resident weight buffers (if b_res)
     const uint32_t stage_base = smem_base + (uint32_t)c.b_res * c.bres_stride;   // b_res = number of resident weight buffers
     const int HW = s.H * s.W;
@@ -389,7 +392,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint32_t bar = smem_u32(&ctl.b_full[0]);
             if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
             __syncwarp();
-            for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+            for (uint32_t blk = lane; blk < (uint32_t)vt * (uint32_t)c.chunks; blk += 32)
                 bulk_load_1d(bres_base + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
             cur_gn = (int)gn;
             switches = 1;
@@ -398,7 +401,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const uint32_t bar1 = smem_u32(&ctl.b_full[1]);
                 if (lane == 0) mbar_arrive_expect_tx(bar1, b_tile_bytes);
                 __syncwarp();
-                for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                for (uint32_t blk = lane; blk < (uint32_t)vt * (uint32_t)c.chunks; blk += 32)
                     bulk_load_1d(bres_base + c.bres_stride + blk * blk_bytes, wblocks + (size_t)b_tile_bytes + (size_t)blk * blk_bytes, blk_bytes, bar1);
                 switches = 2;
             }
@@ -438,7 +441,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     const uint32_t bar = smem_u32(&ctl.b_full[bb]);
                     if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
                     __syncwarp();
-                    for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                    for (uint32_t blk = lane; blk < (uint32_t)vt * (uint32_t)c.chunks; blk += 32)
                         bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
                     cur_gn = (int)gn;
                     ++switches;
@@ -459,12 +462,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     const int pb = c.SR == 2 ? (int)(i >> 1) : (int)i;
                     rb_seg = c.SR == 2 ? (int)(i & 1u) : 0;
                     rb_row0 = 8 * pb - 1;
-                } else if (c.rowbox) rb_row0 = (int)i * c.R - 1;                 // the row above the tile's first row
+                } else if (c.rowbox) rb_row0 = (int)i * c.R - (c.pw ? 0 : 1);    // the row above the tile's first row (pointwise: the first row)
                 else tile_f0 = c.seg_mode ? (int)i * 32 : (int)i * c.R * s.W;    // first flat pixel of the tile
             }
             int my_n = 0, my_f = 0;
             bool have_lane_coords = false;
-            int ch = 0, r = c.nr == 3 ? 1 : 0;
+            int ch = 0, r = (c.nr == 3 || c.pw) ? 1 : 0;   // r = 1: the centre tap (row offset 0)
             for (int ks = 0; ks < kstages; ++ks, ++it) {
                 if (pf && it >= pf_limit) break;
                 // the first pass over the ring finds every stage free
@@ -526,12 +529,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     const uint32_t bar = smem_u32(&ctl.b_full[bb]);
                     if (lane == 0) mbar_arrive_expect_tx(bar, b_tile_bytes);
                     __syncwarp();
-                    for (uint32_t blk = lane; blk < 3u * (uint32_t)c.chunks; blk += 32)
+                    for (uint32_t blk = lane; blk < (uint32_t)vt * (uint32_t)c.chunks; blk += 32)
                         bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
                     cur_gn = (int)gn;
                     ++switches;
                 }
-                if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
+                if (c.nr == 3 || c.pw) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
         };
@@ -641,7 +644,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             uint32_t n, i;
             c.div_spi.divmod(mt * 4u + (uint32_t)pw, n, i);
             const bool img_ok = (int)n < s.N;
-            int ch = 0, r = 0;
+            int ch = 0, r = c.pw ? 1 : 0;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
                 if (it >= (uint32_t)c.stages) {
                     const uint32_t bar = smem_u32(&ctl.empty[stage]);
@@ -678,7 +681,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 if (pending) hand_over(false);
                 pending = true;
                 prev_stage = stage;
-                if (c.nr == 3) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
+                if (c.nr == 3 || c.pw) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
         }
@@ -907,17 +910,23 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const bool edge_dn = c.need_xchg && lane == 31 && wq < 3 && use_right;   // right neighbour is in the next quarter
             for (int k0 = kbeg; k0 < kend; k0 += 8) {
                 float d0[8], d1[8], d2[8];
-                tmem_ld8(t0 + (uint32_t)k0, d0);
-                tmem_ld8(t0 + (uint32_t)(Kt + k0), d1);
-                tmem_ld8(t0 + (uint32_t)(2 * Kt + k0), d2);
+                if (c.pw) {                                // one accumulator per filter, nothing to combine
+                    tmem_ld8(t0 + (uint32_t)k0, d1);
+                } else {
+                    tmem_ld8(t0 + (uint32_t)k0, d0);
+                    tmem_ld8(t0 + (uint32_t)(Kt + k0), d1);
+                    tmem_ld8(t0 + (uint32_t)(2 * Kt + k0), d2);
+                }
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const float up = __shfl_up_sync(0xffffffffu, d0[j], (unsigned)dil);
-                    const float dn = __shfl_down_sync(0xffffffffu, d2[j], (unsigned)dil);
                     float v = d1[j];
-                    if (add_up) v += up;
-                    if (add_dn) v += dn;
+                    if (!c.pw) {
+                        const float up = __shfl_up_sync(0xffffffffu, d0[j], (unsigned)dil);
+                        const float dn = __shfl_down_sync(0xffffffffu, d2[j], (unsigned)dil);
+                        if (add_up) v += up;
+                        if (add_dn) v += dn;
+                    }
                     if (edge_up) v += xchg[buf][wq - 1][0][k0 + j];
                     if (edge_dn) v += xchg[buf][wq + 1][1][k0 + j];
                     if (c.fuse) {
@@ -1002,7 +1011,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
 // When `merge` > 1 that many adjacent groups are presented to the kernel as one group with a
 // block-diagonal filter bank: entries that would mix channels of different groups are zero.
 __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__ w, uint32_t* __restrict__ packed, uint32_t tag) {
-    const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    const int vt = c.pw ? 1 : 3, ht = c.pw ? 1 : 3;   // vertical and horizontal taps
+    const size_t total = (size_t)c.groups * c.NT * vt * c.chunks * c.Np * c.CK;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         packed[0] = tag;
@@ -1016,14 +1026,14 @@ __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__
         const int nb = (int)(t % (c.Np / 8)); t /= (c.Np / 8);
         const int k2 = (int)(t % 2); t /= 2;
         const int k8 = (int)(t % (c.CK / 8)); t /= (c.CK / 8);
-        const int r = (int)(t % 3); t /= 3;
+        const int r = (int)(t % vt); t /= vt;
         const int ch = (int)(t % c.chunks); t /= c.chunks;
         const int nt = (int)(t % c.NT);
         const int g = (int)(t / c.NT);             // merged group
         const int ncol = nb * 8 + n8;
         const int ce = ch * c.CK + k8 * 8 + k2 * 4 + e;   // channel within the merged group
         uint32_t bits = 0;
-        if (ncol < 3 * c.Kt) {
+        if (ncol < ht * c.Kt) {
             const int ss = ncol / c.Kt;
             const int ke = nt * c.Kt + (ncol - ss * c.Kt);  // filter within the merged group
             const int gi = ke / s.Kg;                        // which original group of the merge
@@ -1031,7 +1041,7 @@ __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__
                 const int ko = (g * c.merge + gi) * s.Kg + (ke - gi * s.Kg);
                 // a pointwise (1x1) filter is the centre tap of a 3x3 filter whose other taps are zero
                 const size_t wi = ((size_t)ko) * s.Cg + (ce - gi * s.Cg);
-                const float v = s.KH == 1 ? ((r == 1 && ss == 1) ? w[wi] : 0.f) : w[wi * 9 + r * 3 + ss];
+                const float v = c.pw ? w[wi] : (s.KH == 1 ? ((r == 1 && ss == 1) ? w[wi] : 0.f) : w[wi * 9 + r * 3 + ss]);
                 asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(bits) : "f"(v));
             }
         }
@@ -1163,6 +1173,10 @@ size_t igemm_scratch_bytes(const Shape& s) {
 static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     const Shape s_true = as_3x3(s_any);
     IgemmCfg c;
+    // Pointwise, stride 1: one vertical tap (a third of the stages and MMAs), one accumulator per filter (N = Kt), filter
+    // tiles of up to 128.  (Stride 2 keeps the centre-tap 3x3 form: its row tiles are built around nine staged rows.)
+    c.pw = (s_any.KH == 1 && s_any.KW == 1 && s_any.stride == 1 && C2 == 0) ? 1 : 0;
+    const int vt = c.pw ? 1 : 3;
     const bool fuse = C2 > 0;          // fused grouped + pointwise block: heavy shape, streamed or resident grouped weights
     const IgemmGeom ge = igemm_geom(s_true);
     Shape s = s_true;          // the plane the kernel computes on
@@ -1177,11 +1191,12 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.Kg = s.Kg * c.merge;
     c.CK = (c.Cg % 32 == 0) ? 32 : (c.Cg % 16 == 0 ? 16 : 8);
     c.chunks = c.Cg / c.CK;
-    int kt = c.Kg <= 64 ? c.Kg : 64;
+    const int kt_max = c.pw ? 128 : 64;
+    int kt = c.Kg <= kt_max ? c.Kg : kt_max;
     while (c.Kg % kt != 0 || kt % 8 != 0) kt -= 8;   // largest multiple of 8 dividing Kg, at most 64
     c.Kt = kt;
     c.NT = c.Kg / kt;
-    c.Np = (3 * kt + 15) & ~15;
+    c.Np = (vt * kt + 15) & ~15;
     const int HW = s.H * s.W;
     c.seg_mode = (32 % s.W == 0) && (HW % 32 == 0);
     c.seg_fstep = 32;
@@ -1249,11 +1264,13 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
         c.nr = 3;
         c.wseg = 1;
         c.nseg = 9;
+    } else if (c.rowbox && c.pw) {
+        c.nr = 1;                                        // the tile's own rows, no halo
     } else if (c.rowbox) {
         c.nr = 3;
         c.wseg = c.SR;
         c.nseg = 4 + 2 * c.SR;
-    } else if (s.stride == 1 && s.dilation == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
+    } else if (!c.pw && s.stride == 1 && s.dilation == 1 && s.W % 32 == 0 && s.W <= 64 && (c.seg_mode ? (c.SPI % 4 == 0) : true)) {
         c.nr = 3;
         c.wseg = s.W / 32;
         c.nseg = 4 + 2 * c.wseg;
@@ -1263,13 +1280,14 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     // segments, each loaded with its own row shift -- so a tile costs one barrier round trip instead of three.  Only
     // where a tile straddles images anyway (8x8): 16x16 planes keep their one-box-per-tap copies, which are faster.
     c.tapb = 0;
-    if (!fuse && c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && s.dilation == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
+    if (!fuse && !c.pw && c.seg_mode && c.SPI % 4 != 0 && c.nr == 1 && s.stride == 1 && s.dilation == 1 && c.CK == 32 && c.chunks == 1 && c.NT == 1 && 2 * c.Np <= 256 &&
         3u * (uint32_t)c.Cg * (uint32_t)c.Np * 4u <= 40u * 1024u) {
         c.tapb = 1;
         c.nr = 3;
         c.wseg = 4;
         c.nseg = 12;
     }
+    if (c.pw) c.need_xchg = 0;                          // no horizontal neighbours to exchange
     c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.issuers = c.nacc;                                // MMA-issuing warps: one per accumulator buffer
@@ -1279,7 +1297,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.div_w = make_fastdiv((uint32_t)s.W);
     c.div_nt = make_fastdiv((uint32_t)c.NT);
     const uint32_t blk = (uint32_t)c.Np * c.CK * 4u;
-    const uint32_t b_tile = 3u * c.chunks * blk;
+    const uint32_t b_tile = (uint32_t)vt * c.chunks * blk;
     const uint32_t a_bytes = (uint32_t)c.nseg * c.CK * 128u;
     const uint32_t xchg_bytes = c.need_xchg ? (uint32_t)(kMaxAcc * 4 * 2 * 64 * sizeof(float)) : 0u;
     // Weights of a (group, filter tile) stay resident in shared memory when they fit: two buffers (the next group's
@@ -1311,7 +1329,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     {
         const uint32_t light_total = 110u * 1024u;
         const uint32_t st_bytes = (a_bytes + 1023u) & ~1023u;
-        const int kst = (3 / c.nr) * c.chunks;
+        const int kst = (vt / c.nr) * c.chunks;
         const bool fits = !fuse && 2 * c.Np <= 256 && b_tile <= 40u * 1024u &&
                           c.bres_stride + (uint32_t)(c.tapb ? 1 : (kst == 1 ? 2 : kst + 1)) * st_bytes + xchg_bytes + 1024u <= light_total;
         // the fused block in the same shape: one grouped issuer (warp 1), the second MMA warp issues the pointwise MMAs
@@ -1363,7 +1381,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.d2_bufs = (fuse && c.d2_col + 2 * C2 <= c.tmem_cols) ? 2 : 1;
     c.w2_off = (uint32_t)c.smem_bytes - 1024u;             // behind the stages (and the exchange area)
     c.a2_off = c.w2_off + ((w2_bytes + 1023u) & ~1023u);
-    c.w2_goff = kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    c.w2_goff = kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * vt * c.chunks * c.Np * c.CK;
     if (fuse) {
         c.smem_bytes = (size_t)c.a2_off + a2_bytes + 1024;
         if (c.egroups == 2) c.issuers = 2;
@@ -1436,12 +1454,12 @@ cudaError_t igemm_block_pack(const Shape& s, int C2, const float* w, const float
 
 size_t igemm_packed_bytes(const Shape& s) {
     const IgemmCfg c = igemm_config(s, 148);
-    return kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    return kHeaderBytes + sizeof(float) * (size_t)c.groups * c.NT * (c.pw ? 1 : 3) * c.chunks * c.Np * c.CK;
 }
 
 cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_t st) {
     const IgemmCfg c = igemm_config(s, 148);
-    const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
+    const size_t total = (size_t)c.groups * c.NT * (c.pw ? 1 : 3) * c.chunks * c.Np * c.CK;
     int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
     igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
     return cudaGetLastError();
@@ -1511,7 +1529,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
         const cuuint64_t dims5[5] = {(cuuint64_t)s.W, (cuuint64_t)s.C_in, (cuuint64_t)c.SR, (cuuint64_t)s.H, (cuuint64_t)s.N};
         const cuuint64_t strides5[4] = {HW * 4, c.SR == 2 ? (cuuint64_t)(s.W - 32) * 4 : 128, (cuuint64_t)s.W * 4,
                                         HW * 4 * (cuuint64_t)s.C_in};
-        const cuuint32_t box5[5] = {32, (cuuint32_t)c.CK, (cuuint32_t)(c.s2h ? 1 : c.SR), (cuuint32_t)(c.s2h ? 9 : c.R + 2), 1};
+        const cuuint32_t box5[5] = {32, (cuuint32_t)c.CK, (cuuint32_t)(c.s2h ? 1 : c.SR), (cuuint32_t)(c.s2h ? 9 : (c.pw ? c.R : c.R + 2)), 1};
         const cuuint32_t estr5[5] = {1, 1, 1, 1, 1};
         if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float*>(x), dims5, strides5, box5, estr5,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1551,7 +1569,8 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<6>, igemm_tf32_kernel<7>, igemm_tf32_kernel<8>,
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
-                                                igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>};
+                                                igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
+                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
