@@ -251,7 +251,7 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0,  0}     // fused block, row boxes, two resident banks
          : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1,  0}     // copy-warp producer (14x14, 7x7 planes), tap blocks
          : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1,  0}     // copy-warp producer, one stage per tap
-         : f == 17 ? Family{0,  1,  1,  0,   1,  1,  0,  1,  1, 32, -1, -1,  -1,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, two CTAs per SM
+         : f == 17 ? Family{0,  1,  1,  0,   1,  1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, two CTAs per SM
          : f == 18 ? Family{1,  0,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0, -1,  0,   4, -1,  1,  0,  0,  0,  0,  1}     // pointwise, row boxes
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
 }
@@ -1193,7 +1193,12 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.chunks = c.Cg / c.CK;
     const int kt_max = c.pw ? 128 : 64;
     int kt = c.Kg <= kt_max ? c.Kg : kt_max;
-    while (c.Kg % kt != 0 || kt % 8 != 0) kt -= 8;   // largest multiple of 8 dividing Kg, at most 64
+    while (c.Kg % kt != 0 || kt % 8 != 0) kt -= 8;   // largest multiple of 8 dividing Kg, at most 64 (pointwise: 128)
+    if (c.pw) {
+        // small planes: narrower filter tiles until there is a tile per SM (each re-reads its pixels from L2)
+        const long long px_tiles = ((long long)s.N * s.H * s.W + 127) / 128;
+        while (kt >= 64 && kt % 16 == 0 && (long long)c.groups * (c.Kg / kt) * px_tiles < (long long)sm_count) kt /= 2;
+    }
     c.Kt = kt;
     c.NT = c.Kg / kt;
     c.Np = (vt * kt + 15) & ~15;
