@@ -232,7 +232,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw;
 };
-constexpr int kFamilies = 19;
+constexpr int kFamilies = 20;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -252,7 +252,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1,  0}     // copy-warp producer (14x14, 7x7 planes), tap blocks
          : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1,  0}     // copy-warp producer, one stage per tap
          : f == 17 ? Family{0,  1,  1,  0,   1,  1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, two CTAs per SM
-         : f == 18 ? Family{1,  0,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0, -1,  0,   4, -1,  1,  0,  0,  0,  0,  1}     // pointwise, row boxes
+         : f == 18 ? Family{1,  0,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1, -1, -1,  0, -1,  0,   4, -1,  1,  0,  0,  0,  0,  1}     // pointwise, row boxes
+         : f == 19 ? Family{0,  1,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1, -1, -1,  0, -1,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, one CTA per SM
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1077,6 +1078,10 @@ struct IgemmGeom {
 };
 // A pointwise convolution (1x1, pad 0) runs as the 3x3, pad 1 convolution whose only non-zero tap is the centre one
 // (same output size for either stride); the packing kernel writes the zeros.
+// With stride 1 a pointwise layer has no use for rows at all -- every output pixel reads the input pixel at the same flat
+// position -- so the plane is re-cut into rows the tilings like: 32 wide when H*W is a multiple of 128 (segment tiling,
+// every lane used, whole tiles per image); a width TMA cannot address becomes the widest multiple of 4 up to 32 that
+// divides H*W (14x14 becomes 7x28: no padded copy).
 static Shape as_3x3(const Shape& s) {
     Shape t = s;
     if (s.KH == 1 && s.KW == 1) {
@@ -1084,6 +1089,20 @@ static Shape as_3x3(const Shape& s) {
         t.KW = 3;
         t.pad = 1;
         t.dilation = 1;
+        if (s.stride == 1) {
+            const long long hw = (long long)s.H * s.W;
+            int w = 0;
+            if (s.W % 4 == 0) {
+                if (hw % 128 == 0) w = 32;           // whole tiles per image: one box copy per stage
+            } else {
+                for (int cand = 32; cand >= 4 && w == 0; cand -= 4)
+                    if (hw % cand == 0) w = cand;
+            }
+            if (w != 0 && hw / w < (1 << 30)) {
+                t.W = t.W_out = w;
+                t.H = t.H_out = (int)(hw / w);
+            }
+        }
     }
     return t;
 }
@@ -1164,7 +1183,8 @@ bool igemm_supported(const Shape& s_any) {
     return c.smem_bytes <= (size_t)kMaxDynSmem;   // the smallest pipeline (two stages) must fit
 }
 
-size_t igemm_scratch_bytes(const Shape& s) {
+size_t igemm_scratch_bytes(const Shape& s_any) {
+    const Shape s = as_3x3(s_any);
     const IgemmGeom ge = igemm_geom(s);
     if (!ge.padded || igemm_config(s, kLayoutSMs).soft) return 0;   // copy warps read the real rows: no padded copy
     return sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp;
@@ -1490,7 +1510,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     const float* x = x_in;
     if (c.padded) {
         if (scratch == nullptr) return cudaErrorInvalidValue;
-        const IgemmGeom ge = igemm_geom(s_true);
+        const IgemmGeom ge = igemm_geom(s);
         const size_t planes = (size_t)s.N * s.C_in;
         const size_t total = planes * ge.Hp * (ge.Wp / 4);
         const int blocks = (int)((total + 255) / 256 < (size_t)sm_count * 16 ? (total + 255) / 256 : (size_t)sm_count * 16);
@@ -1506,7 +1526,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
         x = scratch;
     } else if (c.soft) {
         // the kernel walks the virtual padded plane; its copy warps read the real rows of x (the tensor maps go unused)
-        const IgemmGeom ge = igemm_geom(s_true);
+        const IgemmGeom ge = igemm_geom(s);
         s.H = ge.Hp;
         s.W = ge.Wp;
     }
@@ -1575,7 +1595,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
-                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>};
+                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
