@@ -516,7 +516,7 @@ def run_ours(args):
                                  for g in wl.WRN_GROUPS}
         if args.sweep:
             sweep_rows = []
-            for L in wl.sweep_layers(32) + wl.resnext_layers(64) + wl.mobilenetv2_dw_layers(64) + wl.depthwise5x5_layers(64):
+            for L in wl.sweep_layers(32) + wl.resnext_layers(64) + wl.mobilenetv2_dw_layers(64) + wl.depthwise5x5_layers(64) + wl.pointwise_layers(64):
                 ms, v = time_layer(torch, gconv, L, stream, reps=20)
                 sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
             extra["sweep_layers"] = sweep_rows

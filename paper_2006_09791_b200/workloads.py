@@ -163,3 +163,11 @@ def fused_blocks(N: int = 128):
     out.append((Layer("blk64@56", N // 2, 64, 56, 56, 64, groups=16), 64))
     out.append((Layer("blk128@28", N // 2, 128, 28, 28, 128, groups=32), 64))
     return out
+
+
+def pointwise_layers(N: int = 64) -> List[Layer]:
+    """Pointwise (1x1, pad 0, groups = 1) layers: the second half of the paper's G(g) block at the three stages of the
+    WRN-40-2-shaped stack (batch 2N), and the 1x1 layers around a ResNeXt-shaped grouped 3x3 (56x56, 28x28, 14x14)."""
+    mk = lambda n, ci, hw, co, s=1: Layer("pw_%d-%d@%d%s" % (ci, co, hw, "s2" if s == 2 else ""), n, ci, hw, hw, co, 1, 1, s, 0, 1, 1)
+    return [mk(2 * N, 32, 32, 32), mk(2 * N, 64, 16, 64), mk(2 * N, 128, 8, 128), mk(N, 256, 56, 128), mk(N, 128, 56, 256),
+            mk(N, 512, 28, 256), mk(N, 512, 14, 512), mk(N, 256, 56, 512, 2)]

@@ -10,8 +10,8 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
-from paper_2006_09791_b200.workloads import (depthwise5x5_layers, mobilenetv2_dw_layers, resnext_layers, sweep_layers,
-                                             wrn_stack)
+from paper_2006_09791_b200.workloads import (depthwise5x5_layers, mobilenetv2_dw_layers, pointwise_layers, resnext_layers,
+                                             sweep_layers, wrn_stack)
 
 pytestmark = pytest.mark.gpu
 
@@ -87,8 +87,8 @@ def test_group_sweep_at_batch_32(idx):
 
 def _sweep_row_families():
     """The other rows of the bench's sweep table at the batch it times them at: ResNeXt-shaped grouped layers (stride-2
-    row tiles, padded 14x14 and 7x7 planes, tap blocks), MobileNetV2-shaped depthwise 3x3 and depthwise 5x5 layers."""
-    return resnext_layers(64) + mobilenetv2_dw_layers(64)[4:] + depthwise5x5_layers(64)[1:]
+    row tiles, padded 14x14 and 7x7 planes, tap blocks), MobileNetV2-shaped depthwise 3x3 and depthwise 5x5 layers, pointwise layers."""
+    return resnext_layers(64) + mobilenetv2_dw_layers(64)[4:] + depthwise5x5_layers(64)[1:] + pointwise_layers(64)
 
 
 @pytest.mark.parametrize("idx", range(len(_sweep_row_families())))
