@@ -251,9 +251,9 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0,  0}     // fused block, row boxes, two resident banks
          : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1,  0}     // copy-warp producer (14x14, 7x7 planes), tap blocks
          : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1,  0}     // copy-warp producer, one stage per tap
-         : f == 17 ? Family{0,  1,  1,  0,   1,  1,  0,  1,  1, 32, -1, -1,  -1, -1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, two CTAs per SM
-         : f == 18 ? Family{1,  0,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1, -1, -1,  0, -1,  0,   4, -1,  1,  0,  0,  0,  0,  1}     // pointwise, row boxes
-         : f == 19 ? Family{0,  1,  1,  0,  -1, -1,  0,  1,  1, 32, -1, -1,  -1, -1, -1, -1,  0, -1,  0,   4,  0, -1,  0,  0,  0,  0,  1}     // pointwise, segment tilings, one CTA per SM
+         : f == 17 ? Family{0, 1, 1, 0, 1, 1, 0, 1, -1, 32, -1, -1, -1, -1, 2, 2, 0, 0, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, two CTAs per SM
+         : f == 18 ? Family{1, 0, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, -1, 1, 0, 0, 0, 0, 1}     // pointwise, row boxes
+         : f == 19 ? Family{0, 1, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, one CTA per SM
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1193,9 +1193,10 @@ size_t igemm_scratch_bytes(const Shape& s_any) {
 static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     const Shape s_true = as_3x3(s_any);
     IgemmCfg c;
-    // Pointwise, stride 1: one vertical tap (a third of the stages and MMAs), one accumulator per filter (N = Kt), filter
-    // tiles of up to 128.  (Stride 2 keeps the centre-tap 3x3 form: its row tiles are built around nine staged rows.)
-    c.pw = (s_any.KH == 1 && s_any.KW == 1 && s_any.stride == 1 && C2 == 0) ? 1 : 0;
+    // Pointwise: one vertical tap (a third of the stages and MMAs), one accumulator per filter (N = Kt), filter tiles of
+    // up to 128.  Stride 2 computes every pixel and stores the even ones (no stride-2 row tiles: those are built around
+    // nine staged rows).
+    c.pw = (s_any.KH == 1 && s_any.KW == 1 && C2 == 0) ? 1 : 0;
     const int vt = c.pw ? 1 : 3;
     const bool fuse = C2 > 0;          // fused grouped + pointwise block: heavy shape, streamed or resident grouped weights
     const IgemmGeom ge = igemm_geom(s_true);
@@ -1267,7 +1268,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     // (the odd columns still are: TMA cannot skip elements of the innermost dimension).
     c.s2h = 0;
     c.lbo_segs = 1;
-    if (s.stride == 2 && s.W > 8 && s.W <= 62) {
+    if (s.stride == 2 && s.W > 8 && s.W <= 62 && !c.pw) {
         c.s2h = 1;
         c.lbo_segs = 2;
         c.seg_mode = 0;
