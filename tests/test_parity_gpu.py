@@ -157,6 +157,29 @@ def test_pointwise_on_the_tensor_core_variant(cfg):
     check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=41)
 
 
+def test_seeded_random_pointwise_shapes():
+    """Pointwise layers drawn over plane sizes (re-cut planes, odd sizes, one-pixel rows), both strides, groups, narrow and
+    wide filter tiles."""
+    import random
+    rng = random.Random(4242)
+    done = 0
+    while done < 40:
+        g = rng.choice([1, 1, 1, 2, 4, 8])
+        cg = rng.choice([8, 16, 24, 32, 64, 128, 256])
+        kg = rng.choice([8, 16, 32, 40, 64, 80, 128, 256])
+        C, K = g * cg, g * kg
+        if C > 1024 or K > 1024:
+            continue
+        H = rng.choice([1, 4, 7, 8, 9, 14, 15, 16, 17, 28, 31, 32, 33, 56, 57])
+        W = rng.choice([4, 6, 7, 8, 12, 14, 15, 16, 20, 28, 30, 32, 36, 56, 60, 64, 100, 128])
+        stride = rng.choice([1, 1, 2])
+        N = rng.choice([1, 2, 3, 5, 8, 33, 128])
+        while N > 1 and (N * C * H * W > 8e6 or N * K * H * W > 8e6 or N * H * W * C * K > 4e9):
+            N //= 2
+        check_layer(Layer("randpw%d" % done, N, C, H, W, K, 1, 1, stride, 0, 1, g), seed=500 + done)
+        done += 1
+
+
 # Dilated 3x3 (pad = dilation) on the tensor-core variant: vertical taps become shifts by `dilation` rows, horizontal
 # ones lane shifts by `dilation` columns inside a 32-pixel segment, so only planes whose rows divide 32 pixels
 # (after padding the width to a multiple of 4) are taken: 32, 16 and 8 wide, 14 (copy warps) and 7.
