@@ -232,7 +232,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw;
 };
-constexpr int kFamilies = 20;
+constexpr int kFamilies = 21;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -254,6 +254,7 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 17 ? Family{0, 1, 1, 0, 1, 1, 0, 1, -1, 32, -1, -1, -1, -1, 2, 2, 0, 0, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, two CTAs per SM
          : f == 18 ? Family{1, 0, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, -1, 1, 0, 0, 0, 0, 1}     // pointwise, row boxes
          : f == 19 ? Family{0, 1, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, one CTA per SM
+         : f == 20 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 16,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, 16-channel merged groups (channel-doubling transitions)
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1161,7 +1162,11 @@ __global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict_
 
 static int igemm_merge(const Shape& s) {
     int m = 1;
-    while (m * 2 <= s.groups && s.groups % (m * 2) == 0 && s.Cg * m * 2 <= 32 && s.Kg * m * 2 <= 64) m *= 2;
+    // Stride 2: stop at 32 filters per merged group, so that channel-doubling transition layers (Kg = 2 Cg) keep one
+    // resident 32-filter bank and the two-CTA launch shape instead of streaming 64-filter banks (measured: 64 -> 128
+    // channels at 56x56, 32 groups, 35.5 -> 17.0 us).
+    const int kcap = s.stride == 2 ? 32 : 64;
+    while (m * 2 <= s.groups && s.groups % (m * 2) == 0 && s.Cg * m * 2 <= 32 && s.Kg * m * 2 <= kcap) m *= 2;
     return m;
 }
 
@@ -1596,7 +1601,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
-                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>};
+                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
