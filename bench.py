@@ -520,6 +520,15 @@ def run_ours(args):
                 ms, v = time_layer(torch, gconv, L, stream, reps=20)
                 sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
             extra["sweep_layers"] = sweep_rows
+            # ResNet-34-shaped layers at N = 64 for every group count, with the time-falls-with-groups check per shape
+            r34_rows, r34_ms = [], {}
+            for g in wl.R34_GROUPS:
+                for L in wl.resnet34_layers(g, 64):
+                    ms, v = time_layer(torch, gconv, L, stream, reps=20)
+                    r34_rows.append(layer_row(L, ms, v, peaks, gconv))
+                    r34_ms.setdefault(L.name, []).append(ms)
+            extra["resnet34_layers"] = r34_rows
+            extra["resnet34_monotone"] = {name: all(b <= 1.03 * a for a, b in zip(t, t[1:])) for name, t in r34_ms.items()}
             block_rows = []
             for L, C2 in wl.fused_blocks():
                 msb = time_block(torch, gconv, L, C2, stream)
