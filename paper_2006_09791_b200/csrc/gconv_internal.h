@@ -139,6 +139,7 @@ struct IgemmCfg {
     int padded, Hv, Wv;      // the kernel computes on a zero-padded copy of x; valid extent of the plane
     int s2h, lbo_segs;       // stride-2 row tiles (four output rows of one segment, nine staged input rows); segments between M blocks
     int rowbox, SR;          // tile = R whole rows of SR 32-pixel segments each (widths that do not divide 32)
+    int pair, MTr;           // pair tiles: a stage holds the input of two pixel tiles and one set of streamed weights (MT counts pairs, MTr tiles)
     int num_tiles, stages, grid;
     FastDiv div_nt;                   // (group, filter tile) index -> group
     FastDiv div_mt, div_spi, div_w;   // tile -> (group/filter tile, pixel tile); pixel tile -> (image, segment or row block); pixel -> (row, column)

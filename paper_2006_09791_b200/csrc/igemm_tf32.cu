@@ -230,9 +230,9 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
 // instruction stream matters: the 8x8 layers of the WRN stack run 20 % faster on their family than on family 0.
 struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
-        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw;
+        nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 21;
+constexpr int kFamilies = 22;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -255,11 +255,12 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 18 ? Family{1, 0, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, -1, 1, 0, 0, 0, 0, 1}     // pointwise, row boxes
          : f == 19 ? Family{0, 1, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, one CTA per SM
          : f == 20 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 16,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, 16-channel merged groups (channel-doubling transitions)
-                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1};
+         : f == 21 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 16, -1, 64, 192, -1,  1,  1, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0,  0,  1}     // row boxes, 64-filter tiles, streamed weights shared by a pair of pixel tiles
+                  : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
     X(rowbox) X(seg_mode) X(nr) X(need_xchg) X(b_res) X(egroups) X(s2h) X(lbo_segs) X(CK) X(chunks) X(Kt) X(Np) X(NT) X(nacc) X(issuers) \
-    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball) X(soft) X(pw)
+    X(padded) X(nt_fast) X(wseg) X(nseg) X(SR) X(fast4) X(tapb) X(fuse) X(ball) X(soft) X(pw) X(pair)
 
 static bool family_matches(int f, const Shape& s, const IgemmCfg& c) {
     const Family fam = family(f);
@@ -305,7 +306,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         } else if (t >= 8 && t < 8 + kMaxAcc) {
             const int i = t - 8;
             mbar_init(smem_u32(&ctl.tmem_full[i]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[i]), kEpiWarps);
+            mbar_init(smem_u32(&ctl.tmem_empty[i]), c.pair ? 2u * kEpiWarps : (uint32_t)kEpiWarps);   // pair tiles: both groups drain the buffer
             mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
         } else if (t >= 16 && t < 18) {
             const int i = t - 16;
@@ -362,6 +363,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     const int kstages = (vt / c.nr) * c.chunks;
     const uint32_t seg_bytes = (uint32_t)c.CK * 128u;
     const uint32_t a_bytes = (uint32_t)c.nseg * seg_bytes;
+    const uint32_t a_all = c.pair ? 2u * a_bytes : a_bytes;   // pair tiles: the second tile's input sits behind the first's
     const uint32_t blk_bytes = (uint32_t)c.Np * (uint32_t)c.CK * 4u;   // weights of one (chunk, tap)
     const uint32_t b_tile_bytes = (uint32_t)vt * (uint32_t)c.chunks * blk_bytes;   // weights of one (group, filter tile)
     const uint32_t bres_base = smem_base;                                // two resident weight buffers (if b_res)
@@ -456,6 +458,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             // by segment, lane j issuing segment j with its own (image, first pixel).
             const bool whole = c.rowbox || c.fast4;
             int tile_n = 0, tile_f0 = 0, rb_row0 = 0, rb_seg = 0;
+            int tile_n1 = 0, rb_row1 = 0, rb_seg1 = 0;   // pair tiles: the second pixel tile of the pair (row boxes, stride 1)
+            if (c.pair) {
+                mt *= 2u;
+                uint32_t n, i;
+                c.div_spi.divmod(mt + 1u, n, i);         // past the last tile: the image index is out of range, the box reads as zeros
+                tile_n1 = (int)n;
+                rb_row1 = (int)i * c.R - 1;
+            }
             if (whole) {
                 uint32_t n, i;
                 c.div_spi.divmod(c.seg_mode ? mt * 4u : mt, n, i);
@@ -487,13 +497,16 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         else tma_prefetch_4d(&xmap4, lo, chan, 0, tile_n);
                     }
                 } else if (lane == 0) {
-                    mbar_arrive_expect_tx(full, a_bytes + nb);
+                    mbar_arrive_expect_tx(full, a_all + nb);
                     if (box) {
-                        if (c.rowbox) tma_load_5d(a_dst, &xmap4, 0, chan, rb_seg, rb_row0, tile_n, full);   // rows above/below and columns past W: zero fill
+                        if (c.rowbox) {
+                            tma_load_5d(a_dst, &xmap4, 0, chan, rb_seg, rb_row0, tile_n, full);   // rows above/below and columns past W: zero fill
+                            if (c.pair) tma_load_5d(a_dst + a_bytes, &xmap4, 0, chan, rb_seg1, rb_row1, tile_n1, full);
+                        }
                         else if (c.fast4 == 2) tma_load_4d(a_dst, &xmap4, 0, chan, lo >> 5, tile_n, full);   // segments outside the plane read as zeros
                         else tma_load_4d(a_dst, &xmap4, lo, chan, 0, tile_n, full);
                     }
-                    if (nb) bulk_load_1d(a_dst + a_bytes, wtile + (size_t)ks * nb, nb, full);
+                    if (nb) bulk_load_1d(a_dst + a_all, wtile + (size_t)ks * nb, nb, full);
                 }
                 if (!box) {
                     if (!have_lane_coords) {
@@ -712,7 +725,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint32_t view16 = (uint32_t)(c.nr == 3 ? c.wseg : 0) * (seg_bytes >> 4);
             const uint32_t blk16 = blk_bytes >> 4;
             const uint32_t bk16 = b_kstep >> 4;
-            const uint32_t b_in_stage16 = a_bytes >> 4;
+            const uint32_t b_in_stage16 = a_all >> 4;
+            const uint32_t a_pair16 = a_bytes >> 4;   // pair tiles: the second tile's input inside the stage
             uint32_t tcount = 0, switches = 0;
             int stage = 0;
             uint32_t ph = 0;
@@ -773,6 +787,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 #pragma unroll 4
                         for (int k8 = 0; k8 < k8n; ++k8, al += 64u, bl += bk16) {
                             umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc, acc);
+                            if (c.pair) umma_tf32_split(d_tmem + (uint32_t)c.Np, al + a_pair16, a_hi, bl, b_hi, idesc, acc);   // same weights, second tile
                             acc = 1;
                         }
                     }
@@ -828,7 +843,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         for (int tile = tile_first; tile < tile_end;
              tile = tile_next(tile), tpar ^= 1u, buf = (buf + 1 == (uint32_t)c.nacc ? 0u : buf + 1), bph ^= (buf == 0 ? 1u : 0u)) {
             uint32_t gn, mt;
-            if (c.egroups == 2 && tpar != egroup) {           // the other group's tile
+            if (c.egroups == 2 && tpar != egroup && !c.pair) {           // the other group's tile
                 if (c.fuse) {
                     tile_coords(c, (uint32_t)tile, gn, mt);
                     if ((int)gn + 1 == c.n_gn) ++ptiles;
@@ -836,6 +851,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 continue;
             }
             tile_coords(c, (uint32_t)tile, gn, mt);
+            if (c.pair) mt = 2u * mt + egroup;               // pair tiles: group e drains the pair's tile e (accumulator e of the buffer)
             uint32_t n, i;
             int f;
             bool valid;
@@ -856,6 +872,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 }
                 const int col = (h ? s.W - 32 : 0) + lane;
                 valid = row < s.H && col < s.W && (c.SR == 1 || (h == 0 ? col <= 30 : col >= 31));
+                if (c.pair) valid = valid && (int)n < s.N;   // an odd tile count leaves the last pair's second tile empty
                 f = row * s.W + (col < s.W ? col : s.W - 1);
             } else if (c.seg_mode) {
                 c.div_spi.divmod(mt * 4u + (uint32_t)wq, n, i);
@@ -882,7 +899,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const bool add_dn = use_right && lane + dil < 32;
             if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), bph, abort_flag, status, 400 + buf)) break;
             tc_fence_after();
-            const uint32_t t0 = tmem_base + buf * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
+            const uint32_t t0 = tmem_base + (c.pair ? egroup : buf) * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
             // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
             float* yk = y + ((size_t)n * s.C_out + (size_t)gn * Kt + (size_t)kbeg) * OHW + fo;
             // fused block: this lane's slot in the A2 operand (32-pixel block wq, 128-byte row per channel, 32-byte
@@ -1322,6 +1339,23 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.issuers = c.nacc;                                // MMA-issuing warps: one per accumulator buffer
+    // Pair tiles: a filter bank too large to stay resident streams through every CTA's shared memory once per pixel
+    // tile, and that traffic (L2 -> shared memory), not the tensor core, bounds the wide layers.  A stage then holds the
+    // input of TWO pixel tiles and one set of weight blocks; every weight block feeds two MMAs (one per tile, two
+    // accumulators side by side in TMEM), so the weights cross once per 256 pixels.  Stages shrink to 16 channels so
+    // that three of them fit; the two epilogue groups drain the two accumulators at the same time.  The decision uses
+    // only the shape (the packed layout depends on CK).
+    c.pair = 0;
+    c.MTr = c.MT;
+    if (!fuse && !c.pw && c.rowbox && !c.s2h && c.nr == 3 && s.stride == 1 && s.dilation == 1 && c.Kt == 64 && c.Cg % 16 == 0 &&
+        (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u > 144u * 1024u && (long long)c.groups * c.NT * c.MT >= 4LL * kLayoutSMs) {
+        c.pair = 1;
+        c.CK = 16;
+        c.chunks = c.Cg / 16;
+        c.MT = (c.MTr + 1) / 2;
+        c.nacc = 1;
+        c.issuers = 1;
+    }
     c.num_tiles = c.groups * c.NT * c.MT;
     c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)(c.seg_mode ? c.SPI : c.RB));
@@ -1388,7 +1422,8 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
         c.threads += 32 * kSoftWarps;
     }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
-    c.stage_bytes = (a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
+    c.stage_bytes = ((c.pair ? 2u : 1u) * a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
+    if (c.pair) budget_total = 216u * 1024u;          // three 68 KB stages
     const uint32_t budget = budget_total - (uint32_t)c.b_res * c.bres_stride - xchg_bytes;
     int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
@@ -1601,7 +1636,8 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<9>, igemm_tf32_kernel<10>, igemm_tf32_kernel<11>,
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
-                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>};
+                                                igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
+                                                igemm_tf32_kernel<21>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;

@@ -10,8 +10,8 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
-from paper_2006_09791_b200.workloads import (depthwise5x5_layers, mobilenetv2_dw_layers, pointwise_layers, resnext_layers,
-                                             sweep_layers, wrn_stack)
+from paper_2006_09791_b200.workloads import (depthwise5x5_layers, mobilenetv2_dw_layers, pointwise_layers, resnet34_layers,
+                                             resnext_layers, sweep_layers, wrn_stack)
 
 pytestmark = pytest.mark.gpu
 
@@ -83,6 +83,16 @@ def test_group_sweep_at_batch_32(idx):
     x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(78, idx), L.x_dist)
     y, v = _run_full(L, x, w, use_graph=True)
     _check_samples(L, y, x, w, v, _samples(L, 3 if L.groups == 1 else 6, idx))
+
+
+@pytest.mark.parametrize("groups", [1, 2, 8])
+def test_resnet34_layers_at_batch_64(groups):
+    """The ResNet-34-shaped rows of the bench's sweep at the batch it times them at: pair tiles and streamed filter banks
+    (groups 1 and 2), padded 14x14 and 7x7 planes, stride-2 row tiles with wide and narrow groups."""
+    for i, L in enumerate(resnet34_layers(groups, 64)):
+        x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, synth.layer_seed(83, i, groups), L.x_dist)
+        y, v = _run_full(L, x, w, use_graph=(i % 2 == 1))
+        _check_samples(L, y, x, w, v, _samples(L, 3 if groups == 1 else 5, i))
 
 
 def _sweep_row_families():

@@ -99,6 +99,21 @@ def test_large_rowbox_shapes(cfg):
     check_layer(Layer("rowbox", *cfg), seed=11)
 
 
+# Pair tiles (filter banks too large to stay resident, streamed once per two pixel tiles): an odd number of pixel tiles
+# (the last pair's second tile is empty), two and four filter tiles, 28-wide rows (one segment) and 56-/40-wide rows (two
+# segments), a group width that is a multiple of 16 but not of 32, a padded width (54 -> 56), two groups, an even count.
+PAIR_TILE_SHAPES = [
+    (23, 128, 26, 56, 128, 3, 3, 1, 1, 1, 1), (23, 128, 28, 28, 256, 3, 3, 1, 1, 1, 1), (61, 144, 10, 40, 128, 3, 3, 1, 1, 1, 1),
+    (61, 128, 10, 54, 128, 3, 3, 1, 1, 1, 1), (12, 256, 56, 56, 256, 3, 3, 1, 1, 1, 2), (24, 128, 26, 56, 128, 3, 3, 1, 1, 1, 1),
+]
+
+
+@pytest.mark.parametrize("cfg", PAIR_TILE_SHAPES)
+def test_pair_tile_shapes(cfg):
+    err, used = check_layer(Layer("pair", *cfg), seed=3)
+    assert used == gconv.GCONV_VARIANT_IGEMM_TF32
+
+
 # Widths whose rows are not a multiple of 16 bytes, in the configurations where copy warps (cp.async) build the stages
 # instead of TMA: even widths (8-byte copies) and odd ones (4-byte), padded widths 8, 16 and 32, planes that end inside
 # a tile, batches that end inside a tile, many tiles per CTA, several groups per CTA, stride 2 on 7x7 planes.
