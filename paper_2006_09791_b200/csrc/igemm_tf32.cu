@@ -927,6 +927,37 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             }
             const bool edge_up = c.need_xchg && lane == 0 && wq > 0 && use_left;     // left neighbour is in the previous quarter
             const bool edge_dn = c.need_xchg && lane == 31 && wq < 3 && use_right;   // right neighbour is in the next quarter
+            if (c.pair) {
+                // Pair tiles have one accumulator buffer, so the next pair's MMAs wait for this epilogue: read and combine
+                // the warp's 32 filters into registers first, hand the buffer back, and only then store.
+                float v[32];
+#pragma unroll
+                for (int kk = 0; kk < 32; kk += 8) {
+                    float d0[8], d1[8], d2[8];
+                    tmem_ld8(t0 + (uint32_t)(kbeg + kk), d0);
+                    tmem_ld8(t0 + (uint32_t)(Kt + kbeg + kk), d1);
+                    tmem_ld8(t0 + (uint32_t)(2 * Kt + kbeg + kk), d2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float t = d1[j];
+                        const float up = __shfl_up_sync(0xffffffffu, d0[j], 1u);
+                        const float dn = __shfl_down_sync(0xffffffffu, d2[j], 1u);
+                        if (add_up) t += up;
+                        if (add_dn) t += dn;
+                        v[kk + j] = t;
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (valid) *yk = v[j];
+                    yk += OHW;
+                }
+                continue;
+            }
             for (int k0 = kbeg; k0 < kend; k0 += 8) {
                 float d0[8], d1[8], d2[8];
                 if (c.pw) {                                // one accumulator per filter, nothing to combine
