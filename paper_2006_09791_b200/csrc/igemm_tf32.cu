@@ -1173,6 +1173,9 @@ namespace {
 template <typename IDX>
 __global__ void igemm_pad_kernel(const float* __restrict__ x, float* __restrict__ xp, size_t planes, int H, int W, int Hp, int Wp,
                                  FastDiv div_plane, FastDiv div_row) {
+    // the convolution kernel that follows may be scheduled now: its set-up overlaps this copy, and it reads the padded
+    // planes only after its own griddepcontrol.wait (this grid complete and visible)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const size_t per_plane = (size_t)Hp * (Wp / 4);
     const size_t total = planes * per_plane;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
