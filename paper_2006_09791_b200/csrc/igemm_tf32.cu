@@ -232,7 +232,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 22;
+constexpr int kFamilies = 23;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -256,6 +256,7 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 19 ? Family{0, 1, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, one CTA per SM
          : f == 20 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 16,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, 16-channel merged groups (channel-doubling transitions)
          : f == 21 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 16, -1, 64, 192, -1,  1,  1, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0,  0,  1}     // row boxes, 64-filter tiles, streamed weights shared by a pair of pixel tiles
+         : f == 22 ? Family{1,   0,  3,  0,   1,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, one resident bank
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1040,7 +1041,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
                   const IgemmCfg c_in, const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag,
                   const float* __restrict__ x) {
     if constexpr (F == 0) {
-        igemm_tf32_body(xmap, xmap4, s_in, c_in, packed, y, status, tag, x);
+        IgemmCfg c = c_in;
+        c.pair = 0;     // pair tiles always run on their own instantiation (the host refuses anything else)
+        igemm_tf32_body(xmap, xmap4, s_in, c, packed, y, status, tag, x);
     } else {
         constexpr Family fam = family(F);
         IgemmCfg c = c_in;
@@ -1671,10 +1674,11 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
                                                 igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
-                                                igemm_tf32_kernel<21>};
+                                                igemm_tf32_kernel<21>, igemm_tf32_kernel<22>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
+    if (cfg.pair && family(fam).pair != 1) return cudaErrorInvalidValue;   // the generic instantiation has no pair-tile code
     static bool attr_set[64][kFamilies] = {};
     int dev = 0;
     cudaGetDevice(&dev);
