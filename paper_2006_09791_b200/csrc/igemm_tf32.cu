@@ -1401,7 +1401,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     {
         const uint32_t b_any = (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u;
         if (!c.pair && !fuse && !c.pw && c.rowbox && !c.s2h && c.nr == 3 && s.stride == 1 && s.dilation == 1 && c.CK == 32 &&
-            b_any > 40u * 1024u && b_any <= 144u * 1024u && c.MT >= 4 * kLayoutSMs) {
+            b_any > 40u * 1024u && b_any <= 144u * 1024u && c.MT >= 2 * kLayoutSMs) {
             deep_ring = true;
             c.CK = 16;
             c.chunks = c.Cg / 16;
@@ -1426,7 +1426,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
         const uint32_t a_only = (a_bytes + 1023u) & ~1023u;
         if (c.b_res == 1 && c.bres_stride + 2u * a_only + xchg_bytes + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
         // loading a large filter bank up front only pays when a CTA reuses it over several pixel tiles
-        if (!fuse && c.b_res == 1 && b_tile > 40u * 1024u && c.MT < 4 * sm_count) c.b_res = 0;
+        if (!fuse && c.b_res == 1 && b_tile > 40u * 1024u && c.MT < (deep_ring ? 2 : (c.s2h ? 1 : 4)) * sm_count) c.b_res = 0;
     }
     if (fuse && c.b_res == 1 && c.groups * c.NT > 1) c.b_res = 0;   // the group changes every tile: stream, or two buffers
     c.egroups = 2;
