@@ -232,7 +232,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 24;
+constexpr int kFamilies = 26;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -258,6 +258,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 21 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 16, -1, 64, 192, -1,  1,  1, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0,  0,  1}     // row boxes, 64-filter tiles, streamed weights shared by a pair of pixel tiles
          : f == 22 ? Family{1,   0,  3,  0,   1,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, one resident bank
          : f == 23 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 16, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one large resident bank, 16-channel stages
+         : f == 24 ? Family{1,   0,  3,  0,   1,  2,  1,  2,  2, 16, -1, 64, 192, -1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, one resident 64-filter bank, 16-channel stages
+         : f == 25 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 16, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights, 16-channel stages
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -1400,8 +1402,9 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     bool deep_ring = false;
     {
         const uint32_t b_any = (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u;
-        if (!c.pair && !fuse && !c.pw && c.rowbox && !c.s2h && c.nr == 3 && s.stride == 1 && s.dilation == 1 && c.CK == 32 &&
-            b_any > 40u * 1024u && b_any <= 144u * 1024u && c.MT >= 2 * kLayoutSMs) {
+        const bool s1 = !c.s2h && s.stride == 1 && b_any <= 144u * 1024u && c.MT >= 2 * kLayoutSMs;
+        const bool s2 = c.s2h && s.stride == 2 && c.MT >= kLayoutSMs && c.Cg >= 64;   // stride-2 row tiles, resident or streamed banks (one 32-channel chunk: slower)
+        if (!c.pair && !fuse && !c.pw && c.rowbox && c.nr == 3 && s.dilation == 1 && c.CK == 32 && b_any > 40u * 1024u && (s1 || s2)) {
             deep_ring = true;
             c.CK = 16;
             c.chunks = c.Cg / 16;
@@ -1426,7 +1429,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
         const uint32_t a_only = (a_bytes + 1023u) & ~1023u;
         if (c.b_res == 1 && c.bres_stride + 2u * a_only + xchg_bytes + 1024u > (uint32_t)kMaxDynSmem) c.b_res = 0;
         // loading a large filter bank up front only pays when a CTA reuses it over several pixel tiles
-        if (!fuse && c.b_res == 1 && b_tile > 40u * 1024u && c.MT < (deep_ring ? 2 : (c.s2h ? 1 : 4)) * sm_count) c.b_res = 0;
+        if (!fuse && c.b_res == 1 && b_tile > 40u * 1024u && c.MT < (c.s2h ? 1 : (deep_ring ? 2 : 4)) * sm_count) c.b_res = 0;
     }
     if (fuse && c.b_res == 1 && c.groups * c.NT > 1) c.b_res = 0;   // the group changes every tile: stream, or two buffers
     c.egroups = 2;
@@ -1475,7 +1478,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
     c.stage_bytes = ((c.pair ? 2u : 1u) * a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
     if (c.pair) budget_total = 216u * 1024u;          // three 68 KB stages
-    if (deep_ring && c.b_res == 1) budget_total = (uint32_t)kMaxDynSmem - 2048u;
+    if (deep_ring && (c.b_res == 1 || c.s2h)) budget_total = (uint32_t)kMaxDynSmem - 2048u;
     const uint32_t budget = budget_total - (uint32_t)c.b_res * c.bres_stride - xchg_bytes;
     int st = (int)(budget / c.stage_bytes);
     if (st > 8) st = 8;
@@ -1689,7 +1692,8 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<12>, igemm_tf32_kernel<13>,
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
                                                 igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
-                                                igemm_tf32_kernel<21>, igemm_tf32_kernel<22>, igemm_tf32_kernel<23>};
+                                                igemm_tf32_kernel<21>, igemm_tf32_kernel<22>, igemm_tf32_kernel<23>,
+                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
