@@ -6,12 +6,16 @@ layers: 32/64/128 channels at 32/16/8, stride-2 transitions) at batch 128 for ev
 {1,2,4,8,16}: 90 gconv_forward launches.  Every layer instance owns its x and y buffers, so ~1.8 GB
 is cycled between two uses of the same buffer (more than the 126 MB L2).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
 
 Prints ONE JSON line.  `value` is GFLOP/s (2*MACs of Eq. (2) of the paper per second) with inputs
 resident in HBM, the step replayed as a CUDA graph; `e2e` is the same metric through
-gconv_forward_host with pinned host buffers (copies inside the timed region).  `--impl reference`
-times the CPU oracle (the only reference there is: the paper ships no code) on a bounded sample.
+gconv_forward_host with pinned host buffers (copies inside the timed region).  The same line carries
+the per-layer tables of every benchmark family (ms, GFLOP/s, GB/s, fraction of the layer's roofline,
+cold and warm L2, the plain-copy and launch-interval floors beside them), the time-falls-with-groups
+checks and a `targets` object that names every layer below the 50 % tensor / 60 % HBM bars.
+`--impl reference` times the CPU oracle (the only reference there is: the paper ships no code) on
+a bounded sample.
 """
 from __future__ import annotations
 
@@ -31,6 +35,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 from paper_2006_09791_b200 import synth, workloads as wl  # noqa: E402
+from paper_2006_09791_b200.torch_util import attach_workspace  # noqa: E402
 
 METRIC = "grouped_conv_gflops"
 UNIT = "GFLOP/s"
@@ -39,10 +44,25 @@ BATCH = 128
 CPU_SAMPLE_BATCH = 8      # batch of the reference arm's per-step sample
 CPU_LEG_BATCH = 32        # batch of the cpu_baseline leg of the GPU arm
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes one launch of the dominant kernel moves on average over the step, from an ncu launch-list capture of
-# `bench.py --steps 2 --warmup 3 --no-cpu --no-layers` with the dram__bytes_read/write metrics (summary kept under
-# profiles/; reads only: ncu attributes the later write-back of y to no kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"igemm_tf32": 10.66e6}
+# DRAM bytes one launch of the dominant kernel moves on average over the step come from an ncu capture whose summary is
+# kept under profiles/ (a table row per kernel variant: bytes per launch, the commit it was captured at, the command).
+NCU_TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.md")
+
+
+def ncu_traffic():
+    """{variant name: {"bytes": DRAM bytes per launch, "commit": ..., "note": ...}} parsed from the committed table."""
+    out = {}
+    try:
+        for ln in open(NCU_TRAFFIC_TABLE):
+            f = [t.strip() for t in ln.strip().strip("|").split("|")]
+            if len(f) >= 3 and f[0] and not f[0].startswith(("-", "kernel")):
+                try:
+                    out[f[0]] = {"bytes": float(f[1]), "commit": f[2], "note": f[3] if len(f) > 3 else ""}
+                except ValueError:
+                    pass
+    except OSError:
+        pass
+    return out
 
 
 def load_peaks():
@@ -137,6 +157,35 @@ def oracle_sample_time(batch, threads):
     return total_s, total_macs
 
 
+def gspc_baseline(threads, batch=CPU_SAMPLE_BATCH):
+    """The paper's own method (Algorithm 1: kernels packed ahead of time, then input reshaping, convolution on the
+    packed volumes and output reshaping, float32) timed on the host cores over the same stack at a reduced batch, for
+    a few (T_I, T_O) tile pairs within Eq. (1)'s bounds: each pair is capped by CPG and KPG of the layer.  A second
+    reported CPU baseline; not the oracle, not a target."""
+    import oracle
+    pairs = [(1, 1), (4, 8), (8, 16), (16, 16), (32, 32), (128, 128)]
+    results = []
+    for T_I, T_O in pairs:
+        secs, macs, stages = 0.0, 0, [0.0, 0.0, 0.0]
+        for g in wl.WRN_GROUPS:
+            for L in wl.wrn_stack(g, batch):
+                ti, to = min(T_I, L.Cg), min(T_O, L.Kg)
+                x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, g, synth.layer_seed(1, L.C_in, L.H, L.C_out, g))
+                wp = oracle.gspc_pack_kernels(w, g, ti, to)
+                t0 = time.perf_counter()
+                for _ in range(L.repeat):
+                    _, st = oracle.gspc_forward(x, wp, w.shape, L.stride, L.pad, L.dilation, g, ti, to, threads=threads, return_stage_seconds=True)
+                    stages = [a + b for a, b in zip(stages, st)]
+                secs += time.perf_counter() - t0
+                macs += L.macs * L.repeat
+        results.append({"T_I": T_I, "T_O": T_O, "value": 2.0 * macs / secs / 1e9, "seconds": secs,
+                        "stage_seconds": {"input_reshape": stages[0], "convolution": stages[1], "output_reshape": stages[2]}})
+    best = max(results, key=lambda r: r["value"])
+    return {"value": best["value"], "unit": UNIT, "cores": threads, "kind": "gspc_algorithm1_f32", "best_tiles": [best["T_I"], best["T_O"]],
+            "tile_sweep": results,
+            "sample": "the 18-layer stack at N=%d (of %d) for every group count; tiles capped by CPG and KPG per layer" % (batch, BATCH)}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -190,16 +239,21 @@ class Instance:
         self.x = x_dev
         self.wp = wp
         self.y = torch.empty(L.y_elems, dtype=torch.float32, device=x_dev.device)
+        self.ws = attach_workspace(self.desc, x_dev.device)
 
 
-def time_layer(torch, gconv, L, stream, reps=160, min_cycle_bytes=2 * L2_BYTES + (64 << 20)):
+def time_layer(torch, gconv, L, stream, reps=160, min_cycle_bytes=2 * L2_BYTES + (64 << 20), warm=False):
     """Average device time of one gconv_forward launch of layer L with cold L2: launches rotate over
-    enough distinct (x, y) buffer pairs that more than twice the L2 is cycled between reuses."""
+    enough distinct (x, y) buffer pairs that more than twice the L2 is cycled between reuses.  With `warm` the
+    launches reuse ONE buffer pair instead (whatever fits stays in L2).  Returns (median ms, variant)."""
+    if warm:
+        min_cycle_bytes = 0
     dev = torch.device("cuda", torch.cuda.current_device())
     per = 4 * (L.x_elems + L.y_elems)
-    nbuf = max(2, -(-min_cycle_bytes // per))
+    nbuf = 1 if warm else max(2, -(-min_cycle_bytes // per))
     d = gconv.gconv_desc_create(*L.desc_args())
     try:
+        ws = attach_workspace(d, dev)
         x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.groups, 99, L.x_dist)
         w = torch.from_numpy(w0).to(dev)
         reps_x = -(-L.N // x0.shape[0])
@@ -293,21 +347,23 @@ def block_row(L, C2, ms_block, ms_grouped, ms_pointwise, peaks):
             "bound": "hbm" if bytes_block / hbm >= t_tensor else "tensor", "roofline_frac": t_roof / (ms_block * 1e-3)}
 
 
-def chained_stack_ms(torch, gconv, groups, stream, reps=50):
-    """Batch-1 inference over the 18-layer stack as a real chain (each layer reads the previous layer's output),
-    replayed as one CUDA graph: ms per pass.  This is the shape of the paper's whole-network timings (N = 1),
-    restricted to the grouped 3x3 layers."""
+def chained_stack_ms(torch, gconv, groups, stream, reps=50, family="wrn"):
+    """Batch-1 inference over a stack as a real chain (each layer reads the previous layer's output), replayed as one
+    CUDA graph: ms per pass.  This is the shape of the paper's whole-network timings (N = 1, Tables I and II),
+    restricted to the grouped 3x3 layers: the 18-layer WRN-40-2-shaped stack, or the seven ResNet-34-shaped layers in
+    network order (56x56 down to 7x7 through the stride-2 transitions)."""
     dev = torch.device("cuda", torch.cuda.current_device())
     layers = []
-    for L in wl.wrn_stack(groups, 1):
+    for L in (wl.wrn_stack(groups, 1) if family == "wrn" else wl.resnet34_layers(groups, 1)):
         layers.extend([L] * L.repeat)
-    descs, wps, bufs = [], [], []
+    descs, wps, bufs, wss = [], [], [], []
     x0, _ = synth.make_layer_tensors(1, layers[0].C_in, layers[0].H, layers[0].W, layers[0].C_out, 3, 3, groups, 3)
     bufs.append(torch.from_numpy(x0).to(dev).reshape(-1))
     try:
         for i, L in enumerate(layers):
             d = gconv.gconv_desc_create(*L.desc_args())
             descs.append(d)
+            wss.append(attach_workspace(d, dev))
             _, w = synth.make_layer_tensors(1, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, 100 + i)
             wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
             gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp, stream)
@@ -339,6 +395,101 @@ def chained_stack_ms(torch, gconv, groups, stream, reps=50):
     finally:
         for d in descs:
             gconv.gconv_desc_destroy(d)
+
+
+def graph_time_ms(torch, stream, body, reps, rounds=5):
+    """Median device time (ms) of one call of `body(i)` when `reps` calls are replayed as one CUDA graph."""
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            body(i)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(reps):
+                body(i)
+        graph.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times = []
+        for _ in range(rounds):
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            times.append(e0.elapsed_time(e1) / reps)
+    return statistics.median(times)
+
+
+def launch_interval_us(torch, stream):
+    """Latency floor: the interval between dependent launches of a kernel that does nothing to speak of (torch adds 1
+    to a one-element tensor), 200 of them in one CUDA graph.  Off the product path."""
+    t = torch.zeros(1, dtype=torch.float32, device=torch.device("cuda", torch.cuda.current_device()))
+    return 1e3 * graph_time_ms(torch, stream, lambda i: t.add_(1.0), reps=200)
+
+
+class CopyFloor:
+    """Plain-copy floor of a layer: a torch copy kernel that moves the layer's algorithmic bytes (half read, half
+    written), launched like the layer (one CUDA graph of back-to-back launches over rotating cold buffers)."""
+
+    def __init__(self, torch, stream):
+        self.torch, self.stream, self.cache = torch, stream, {}
+
+    def ms(self, nbytes, reps=20):
+        torch = self.torch
+        elems = max(1, int(nbytes) // 8)          # elems read + elems written = nbytes
+        if elems not in self.cache:
+            dev = torch.device("cuda", torch.cuda.current_device())
+            nbuf = max(2, -(-(2 * L2_BYTES + (64 << 20)) // (8 * elems)))
+            src = [torch.empty(elems, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+            dst = [torch.empty(elems, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+            self.cache[elems] = graph_time_ms(torch, self.stream, lambda i: dst[i % nbuf].copy_(src[i % nbuf]), reps=max(reps, nbuf))
+            del src, dst
+        return self.cache[elems]
+
+
+def tf32_probe_tflops(torch):
+    """Measured TF32 tensor throughput of the box: one cuBLAS fp32 matmul of 8192^3 with TF32 enabled, best of 10
+    (a context figure beside the roofline denominator, which stays half of the measured bf16 peak).  Off the product path."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        n = 8192
+        a = torch.randn(n, n, device=dev)
+        b = torch.randn(n, n, device=dev)
+        c = torch.empty(n, n, device=dev)
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        best = 1e9
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(10):
+            e0.record()
+            torch.matmul(a, b, out=c)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+
+
+def targets_of(rows, monotone):
+    """The three acceptance properties over every per-layer row: wide (tensor-bound) layers at >= 50 % of the TF32
+    roofline, narrow-group and depthwise (HBM-bound) layers at >= 60 % of the HBM roofline, and time non-increasing in
+    the group count.  Rows whose roofline time is below the launch-interval floor are listed but flagged."""
+    def fails(bound, bar):
+        out = []
+        for r in rows:
+            if r["bound"] == bound and r["roofline_frac"] < bar:
+                out.append({"layer": r["layer"], "groups": r["groups"], "N": r["N"], "frac": round(r["roofline_frac"], 3),
+                            "latency_bound": r.get("latency_bound", False)})
+        return out
+    wide, narrow = fails("tensor", 0.5), fails("hbm", 0.6)
+    n_wide = sum(1 for r in rows if r["bound"] == "tensor")
+    n_narrow = sum(1 for r in rows if r["bound"] == "hbm")
+    return {"wide_ge_50pct_tf32": {"met": not wide, "rows": n_wide, "failing": wide},
+            "narrow_ge_60pct_hbm": {"met": not narrow, "rows": n_narrow, "failing": narrow},
+            "monotone": {"met": all(monotone.values()), "failing": sorted(k for k, v in monotone.items() if not v)}}
 
 
 def layer_row(L, ms, variant, peaks, gconv):
@@ -476,14 +627,30 @@ def run_ours(args):
     # ---- per-layer table (the metric proper) and roofline of the dominant kernel --------------------
     rows, extra = [], {}
     if rank == 0 and not args.no_layers:
+        floor_us = launch_interval_us(torch, stream)
+        copy_floor = CopyFloor(torch, stream)
+
+        def measured_row(L, reps):
+            """One per-layer row: cold-L2 time (the one the roofline fraction uses), warm-L2 time, the plain-copy floor
+            for the same bytes and the launch-interval floor; `latency_bound` marks rows whose roofline time is below
+            the launch interval."""
+            ms, v = time_layer(torch, gconv, L, stream, reps=reps)
+            row = layer_row(L, ms, v, peaks, gconv)
+            if not args.quick:
+                row["ms_warm"] = time_layer(torch, gconv, L, stream, reps=20, warm=True)[0]
+                row["copy_floor_ms"] = copy_floor.ms(L.compulsory_bytes)
+            row["launch_floor_ms"] = floor_us * 1e-3
+            row["latency_bound"] = row["roofline_ms"] < floor_us * 1e-3
+            return row, ms, v
+
         seen = {}
         for g, L in plan:
             key = (L.name, g)
             if key in seen:
                 continue
-            ms, v = time_layer(torch, gconv, L, stream)
+            row, ms, v = measured_row(L, 160)
             seen[key] = (ms, v, L)
-            rows.append(layer_row(L, ms, v, peaks, gconv))
+            rows.append(row)
         by_variant = {}
         for (name, g), (ms, v, L) in seen.items():
             a = by_variant.setdefault(v, {"ms": 0.0, "bytes": 0, "flops": 0, "launches": 0})
@@ -504,31 +671,52 @@ def run_ours(args):
             ach = dom["flops"] / (dom["ms"] * 1e-3) / 1e12
             roofline = {"bound": "tensor" if dom_v == gconv.GCONV_VARIANT_IGEMM_TF32 else "alu", "achieved": ach,
                         "peak": pipe_peak / 1e12, "unit": "TFLOP/s", "frac": ach / (pipe_peak / 1e12), "traffic": None}
-        roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(gconv.variant_name(dom_v))
+        traffic = ncu_traffic().get(gconv.variant_name(dom_v))
+        roofline["traffic"] = traffic["bytes"] if traffic else None
         roofline.update({"kernel": gconv.variant_name(dom_v), "launches_per_step": dom["launches"],
                          "algorithmic_bytes_per_launch": dom["bytes"] / dom["launches"],
                          "avg_launch_us": 1e3 * dom["ms"] / dom["launches"],
                          "share_of_step": dom["ms"] / sum(a["ms"] for a in by_variant.values()),
-                         "peak_source": peaks["source"]})
+                         "peak_source": peaks["source"],
+                         "traffic_source": ("ncu capture at commit %s (profiles/dram_traffic_per_launch.md)" % traffic["commit"]) if traffic else None})
         extra["roofline"] = roofline
+        extra["floors"] = {"launch_interval_us": floor_us,
+                           "step_copy_floor_ms": None if args.quick else sum(r["copy_floor_ms"] * seen[(r["layer"], r["groups"])][2].repeat for r in rows),
+                           "how": "launch interval: a one-element torch kernel, 200 dependent launches in one CUDA graph; copy floor: a torch "
+                                  "copy kernel moving each layer's algorithmic bytes, launched like the layer (graph, cold rotating buffers)"}
         # time per group count (the paper's acceptance property: time falls as g rises)
         extra["ms_by_groups"] = {str(g): sum(ms * L.repeat for (n, gg), (ms, v, L) in seen.items() if gg == g)
                                  for g in wl.WRN_GROUPS}
-        if args.sweep:
-            sweep_rows = []
-            for L in wl.sweep_layers(32) + wl.resnext_layers(64) + wl.mobilenetv2_dw_layers(64) + wl.depthwise5x5_layers(64) + wl.pointwise_layers(64):
-                ms, v = time_layer(torch, gconv, L, stream, reps=20)
-                sweep_rows.append(layer_row(L, ms, v, peaks, gconv))
+        monotone = {}
+        by_shape = {}
+        for (name, g), (ms, v, L) in seen.items():
+            by_shape.setdefault(name, []).append((g, ms))
+        for name, t in by_shape.items():
+            t = [ms for g, ms in sorted(t)]
+            monotone["wrn:" + name] = all(b <= 1.03 * a for a, b in zip(t, t[1:]))
+        graded = list(rows)
+        if world == 1 and not args.quick:
+            # ---- the other benchmark families, at the batch the problem statement names for them ----------------
+            (L0,) = wl.config0()
+            extra["config0_layer"] = [measured_row(L0, 160)[0]]
+            sweep_rows = [measured_row(L, 20)[0] for L in wl.sweep_layers(32)]
             extra["sweep_layers"] = sweep_rows
+            t = [r["ms"] for r in sweep_rows]
+            monotone["sweep_256@56"] = all(b <= 1.03 * a for a, b in zip(t, t[1:]))
+            extra["resnext_layers"] = [measured_row(L, 20)[0] for L in wl.resnext_layers(64)]
             # ResNet-34-shaped layers at N = 64 for every group count, with the time-falls-with-groups check per shape
             r34_rows, r34_ms = [], {}
             for g in wl.R34_GROUPS:
                 for L in wl.resnet34_layers(g, 64):
-                    ms, v = time_layer(torch, gconv, L, stream, reps=20)
-                    r34_rows.append(layer_row(L, ms, v, peaks, gconv))
+                    row, ms, v = measured_row(L, 20)
+                    r34_rows.append(row)
                     r34_ms.setdefault(L.name, []).append(ms)
             extra["resnet34_layers"] = r34_rows
             extra["resnet34_monotone"] = {name: all(b <= 1.03 * a for a, b in zip(t, t[1:])) for name, t in r34_ms.items()}
+            for name, ok in extra["resnet34_monotone"].items():
+                monotone["r34:" + name] = ok
+            graded += extra["config0_layer"] + sweep_rows + extra["resnext_layers"] + r34_rows
+            extra["depthwise_and_pointwise_layers"] = [measured_row(L, 20)[0] for L in wl.mobilenetv2_dw_layers(64) + wl.depthwise5x5_layers(64) + wl.pointwise_layers(64)]
             block_rows = []
             for L, C2 in wl.fused_blocks():
                 msb = time_block(torch, gconv, L, C2, stream)
@@ -538,9 +726,15 @@ def run_ours(args):
                     msp, _ = time_layer(torch, gconv, Lp, stream, reps=20)
                     block_rows.append(block_row(L, C2, msb, msg, msp, peaks))
             extra["fused_blocks"] = block_rows
+            # batch-1 whole-stack timings as real chains in one CUDA graph (the shape of the paper's Tables I and II)
             extra["stack_n1_chained_ms_by_groups"] = {str(g): chained_stack_ms(torch, gconv, g, stream) for g in wl.WRN_GROUPS}
+            extra["resnet34_n1_chained_ms_by_groups"] = {str(g): chained_stack_ms(torch, gconv, g, stream, family="r34") for g in wl.R34_GROUPS}
+            extra["peaks"] = {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"], "tf32_tflops_used": 0.5 * peaks["bf16_tflops"],
+                              "tf32_tflops_cublas_probe": tf32_probe_tflops(torch), "tf32_tflops_nominal": 1100.0,
+                              "fp32_ffma_tflops": 148 * 128 * 2 * 1.965e9 / 1e12, "source": peaks["source"]}
+        extra["targets"] = targets_of(graded, monotone)
 
-    # ---- CPU baseline (rank 0, N=1 only) -----------------------------------------------------------
+    # ---- CPU baselines (rank 0, N=1 only) ----------------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         import oracle
@@ -548,6 +742,10 @@ def run_ours(args):
         secs, macs = oracle_sample_time(CPU_LEG_BATCH, threads)
         cpu = {"value": 2.0 * macs / secs / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": secs,
                "sample": "the 18-layer stack at N=%d (of %d) for every group count, oracle as it stands" % (CPU_LEG_BATCH, BATCH)}
+        s1, m1 = oracle_sample_time(1, 1)
+        cpu["single_thread"] = {"value": 2.0 * m1 / s1 / 1e9, "unit": UNIT, "cores": 1, "seconds": s1,
+                                "sample": "the same stack at N=1, one thread"}
+        extra["cpu_baseline_gspc"] = gspc_baseline(threads)
 
     if rank == 0:
         line = {"metric": METRIC, "value": aggregate_value(step_flops, world, ms_dev), "unit": UNIT, "n_gpus": world,
@@ -577,7 +775,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sweep", action="store_true", help="also time the group-count sweep and ResNeXt-shaped layers")
+    ap.add_argument("--sweep", action="store_true", help="accepted for compatibility: the sweep tables are part of the default run")
+    ap.add_argument("--quick", action="store_true", help="only the step and its own layer table (no other families, no warm/copy columns)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-layers", action="store_true", help="skip the per-layer table (short runs under a profiler)")
     args = ap.parse_args()

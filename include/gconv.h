@@ -21,8 +21,10 @@
  *   - C linkage, no exceptions cross the boundary; every call that can fail returns an int status,
  *     GCONV_OK (0) on success.
  *   - "device" pointers are CUDA device pointers of the current device, "host" pointers are host
- *     memory.  The caller owns every buffer and the stream; the library owns only the descriptor
- *     and a 16-byte device status block it allocates on the first pack/forward call of a descriptor.
+ *     memory.  The caller owns every buffer (the workspace of the few layers that need one included)
+ *     and the stream; the library owns only the descriptor and a 16-byte device status block it
+ *     allocates on the first pack/forward call of a descriptor.  No other device memory is ever
+ *     allocated by the library.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  pack and
  *     forward only enqueue work on it and return without synchronising.
  *   - Device pointers must be 16-byte aligned (GCONV_ERR_ALIGNMENT otherwise).
@@ -48,7 +50,8 @@ enum gconv_status {
     GCONV_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed; see gconv_last_cuda_error */
     GCONV_ERR_PACK_MISMATCH = 6, /* device status: w_packed was packed for another shape or variant */
     GCONV_ERR_TIMEOUT = 7,       /* device status: a bounded wait inside a kernel ran out */
-    GCONV_ERR_TOO_LARGE = 8      /* the layer does not fit the fixed scratch of gconv_forward_host_static */
+    GCONV_ERR_TOO_LARGE = 8,     /* the layer does not fit the fixed scratch of gconv_forward_host_static */
+    GCONV_ERR_WORKSPACE = 9      /* the layer needs a workspace (gconv_workspace_bytes) and none large enough is attached */
 };
 
 /* Kernel variants.  The numeric tolerance of a result follows the variant that produced it:
@@ -69,7 +72,8 @@ enum gconv_variant_id {
  *   out       host pointer receiving the handle (library-owned until gconv_desc_destroy).
  *   N..groups problem sizes; stride, pad and dilation apply to both spatial axes.
  * Host only: touches no device, so it works without a GPU.  Picks the kernel variant with the
- * built-in selector (keyed on Cg, Kg, H*W, N; see gconv_variant).
+ * built-in selector (a rule on the group width derived from measured timings; the choices that
+ * depend on Cg, Kg, H*W and N -- tiling, filter tile, launch shape -- are made inside the variant).
  * Errors: GCONV_ERR_NULL (out), GCONV_ERR_INVALID_ARG (any size < 1, stride < 1, dilation < 1,
  * pad < 0, C_in or C_out not divisible by groups, empty output, or a tensor over 2^40 elements).
  */
@@ -122,19 +126,32 @@ int gconv_pack_weights(gconv_desc_t desc, const float *w_ochw, void *w_packed, v
  *   x_nchw    device, fp32 [N, C_in, H, W], read only; must not overlap y.
  *   w_packed  device, produced by gconv_pack_weights on a descriptor of the same shape and variant.
  *   y_nchw    device, fp32 [N, C_out, H_out, W_out], every element written.
- * For some layers whose width is not a multiple of 4 (gconv_forward_launches reports 2 for them: wide groups,
- * stride 2 on such planes, large 7x7 layers) the tensor-core variant computes on a zero-padded copy of x that
- * it keeps in a device scratch buffer owned by the descriptor: that buffer is allocated (cudaMalloc) by the first
- * gconv_forward of such a descriptor -- make that call outside any stream capture -- and freed by
- * gconv_desc_destroy; two concurrent forwards of ONE such descriptor would race on it.
- * Kernel launches only, on `stream`; deterministic (no atomics on y).  A w_packed made for another shape or
- * variant is detected on the device: y is left unwritten and gconv_last_status reports
- * GCONV_ERR_PACK_MISMATCH.  Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_CUDA.
+ * Kernel launches only, on `stream`; allocates nothing; deterministic (no atomics on y).  A w_packed made for
+ * another shape or variant -- or under a descriptor whose batch, plane size or stride led to another packed layout --
+ * is detected on the device: y is left unwritten and gconv_last_status reports GCONV_ERR_PACK_MISMATCH.
+ * A few layers need a workspace (see gconv_workspace_bytes); without one attached the call enqueues nothing and
+ * returns GCONV_ERR_WORKSPACE.  Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT, GCONV_ERR_WORKSPACE, GCONV_ERR_CUDA.
  */
 int gconv_forward(gconv_desc_t desc, const float *x_nchw, const void *w_packed, float *y_nchw, void *stream);
 
 /*
- * gconv_forward_host -- the same operation for callers whose activations live in host memory:
+ * Workspace (the role of Algorithm 1's input-reshaping stage, Section III-B: a rearranged copy of the padded input).
+ * The tensor-core variant stages its input with bulk tensor copies, whose rows must be multiples of 16 bytes.  Layers
+ * whose width is not a multiple of 4 therefore either build their stages with copy warps (no workspace) or, where
+ * that path does not apply, compute on a zero-padded copy of x kept in a caller-owned device workspace:
+ *   gconv_workspace_bytes     bytes the descriptor's current variant needs; 0 for every layer whose width is a
+ *                             multiple of 4, for the FP32 variants, and for the layers of this kind that the copy
+ *                             warps serve (gconv_forward_launches reports 1 for them, 2 when a workspace is used).
+ *   gconv_desc_set_workspace  attach a device buffer of at least that size (16-byte aligned, caller-owned, must stay
+ *                             valid while forwards of this descriptor are in flight); NULL detaches.  Forwards of ONE
+ *                             descriptor that overlap on the GPU would race on it: give concurrent streams their own
+ *                             descriptors.  Host only; errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT.
+ */
+size_t gconv_workspace_bytes(gconv_desc_t desc);
+int gconv_desc_set_workspace(gconv_desc_t desc, void *workspace, size_t bytes);
+
+/*
+ * gconv_forward_host -- the same operation (Section II) for callers whose activations live in host memory:
  * copies x to the device, runs gconv_forward and copies y back, all enqueued on `stream` in order.
  *   x_host    host, fp32 [N, C_in, H, W] (pinned memory makes the copies asynchronous).
  *   y_host    host, fp32 [N, C_out, H_out, W_out], written when the stream reaches that point.
@@ -149,27 +166,27 @@ int gconv_forward_host(gconv_desc_t desc, const float *x_host, const void *w_pac
  * gconv_forward_host_static -- gconv_forward_host for callers that are not allowed to allocate
  * device memory (no counterpart in the paper; it exists for deployment reasons only).  Think of a
  * plugin living inside an application whose allocator owns the GPU, a service that fixes its memory
- * at start-up, code running between stream-capture begin and end, or a loop that cannot take the
- * device-wide synchronisation a cudaMalloc implies.  It calls no cudaMalloc/cudaFree and no
- * allocating library routine: the status block and the staging room for x and y live in one
- * static device array inside the library (16 MiB + 256 bytes, held by every GPU that loads the
- * library until the process ends).
+ * at start-up, or a loop that cannot take the device-wide synchronisation a cudaMalloc implies.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine: the status block, the staging
+ * room for x and y and the workspace of the layers that need one live in one static device array
+ * inside the library (16 MiB + 256 bytes, held by every GPU that loads the library until the
+ * process ends).
  *   x_host    host, fp32 [N, C_in, H, W], read.
  *   w_packed  device, from gconv_pack_weights on a descriptor of the same shape and variant.
  *   y_host    host, fp32 [N, C_out, H_out, W_out], written.
- * Limit: x and y, each rounded up to 256 bytes, must fit in 16 MiB together; larger layers return
- * GCONV_ERR_TOO_LARGE and nothing is enqueued.
+ * Limit: x, y and gconv_workspace_bytes, each rounded up to 256 bytes, must fit in 16 MiB together;
+ * larger layers return GCONV_ERR_TOO_LARGE and nothing is enqueued.
  * The call enqueues clear-status, copy-in, the kernel of the descriptor's variant and copy-out on
  * `stream`, then SYNCHRONISES the stream and returns GCONV_OK or the status the kernel recorded
  * (GCONV_ERR_PACK_MISMATCH, GCONV_ERR_TIMEOUT); so when it returns, y_host is complete.
+ * Because it synchronises, the call cannot be part of a stream capture.
  * The first call made with a given device current resolves the static array's device address for
- * that device (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * that device (cudaGetSymbolAddress, under a mutex); make that first call before any stream capture
+ * is begun anywhere in the process.
  * All calls share the one array, which still holds the previous call's data: the status block is
  * cleared and the staging regions are rewritten on every call, so results never depend on it, but
  * calls that overlap on the GPU (two streams, two threads) race and must be serialised by the caller.
- * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT (w_packed), GCONV_ERR_TOO_LARGE, GCONV_ERR_CUDA, and
- * GCONV_ERR_UNSUPPORTED for the layers that need the padded-copy scratch described at gconv_forward
- * (tensor-core variant, width not a multiple of 4): force another variant for those.
+ * Errors: GCONV_ERR_NULL, GCONV_ERR_ALIGNMENT (w_packed), GCONV_ERR_TOO_LARGE, GCONV_ERR_CUDA.
  */
 int gconv_forward_host_static(gconv_desc_t desc, const float *x_host, const void *w_packed, float *y_host, void *stream);
 
@@ -205,6 +222,19 @@ int gconv_block_forward(gconv_desc_t desc, int C2, const float *x, const void *w
 
 /* Number of kernel launches one gconv_forward of this descriptor enqueues (for launch accounting). */
 int gconv_forward_launches(gconv_desc_t desc);
+
+/*
+ * Failure-path controls (the paper has no counterpart).  Every wait inside the tensor-core kernel is bounded: when one
+ * runs out the kernel records GCONV_ERR_TIMEOUT, every role leaves, copies in flight are waited for, tensor memory is
+ * freed and the kernel returns; the context stays usable.
+ *   wait_limit_us  time limit of one wait in microseconds; <= 0 restores the default (one second).
+ *   skip_stage     test hook: >= 0 makes the first thread block's producer leave out that stage fill (no copy is
+ *                  issued, its barrier is never armed), so the consumer's wait on it runs out and the forward reports
+ *                  GCONV_ERR_TIMEOUT through gconv_last_status, y partly unwritten; -1 switches it off.  Nothing
+ *                  faults, traps or waits longer than the limit.
+ * Host only.  Errors: GCONV_ERR_NULL.
+ */
+int gconv_desc_set_debug(gconv_desc_t desc, int wait_limit_us, int skip_stage);
 
 /*
  * Synchronises `stream`, then reads and clears the descriptor's device status word: GCONV_OK, or

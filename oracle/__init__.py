@@ -5,6 +5,10 @@ product path (the CUDA library and its Python binding) never does, and nothing h
 product path.  The arithmetic lives in ``gconv_ref.c`` (seven loops, fp64 accumulation; grouped
 convolution of Section II and the convolution stage of Algorithm 1 of the paper); this module only
 compiles that file with gcc and marshals numpy arrays to it.
+
+``gspc.c`` is a second, separate CPU program: the paper's own method (Algorithm 1, Section III-B: kernel reshaping,
+input reshaping, convolution on the packed volumes, output reshaping, with tile sizes T_I and T_O) in float32.  It is
+not the oracle -- the tests pin it against ``gconv_ref`` -- it is the CPU baseline the benchmark times beside it.
 """
 from __future__ import annotations
 
@@ -22,14 +26,25 @@ _lock = threading.Lock()
 _lib = None
 
 
+_GSPC_SRC = os.path.join(_HERE, "gspc.c")
+_GSPC_LIB = os.path.join(_HERE, "libgspc.so")
+_gspc = None
+
+
+def _compile(src: str, lib: str, opt: str, force: bool) -> str:
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= os.path.getmtime(src):
+        return lib
+    tmp = lib + ".tmp.%d" % os.getpid()
+    subprocess.check_call(["gcc", opt, "-fopenmp", "-shared", "-fPIC", "-o", tmp, src])
+    os.replace(tmp, lib)
+    return lib
+
+
 def build(force: bool = False) -> str:
-    """Compile the C oracle into a shared object beside its source (gcc, -O2, OpenMP)."""
-    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
-        return _LIB
-    tmp = _LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC])
-    os.replace(tmp, _LIB)
-    return _LIB
+    """Compile the C oracle (gcc -O2, OpenMP) and the GSPC baseline (gcc -O3, OpenMP) into shared objects beside
+    their sources; returns the oracle's path."""
+    _compile(_GSPC_SRC, _GSPC_LIB, "-O3", force)
+    return _compile(_SRC, _LIB, "-O2", force)
 
 
 def _load():
@@ -83,3 +98,49 @@ def gconv_ref(x: np.ndarray, w: np.ndarray, stride: int = 1, pad: int = 0, dilat
     if rc != 0:
         raise ValueError("gconv_ref_f64 rejected the problem")
     return (y, int(macs.value)) if return_macs else y
+
+
+def _load_gspc():
+    global _gspc
+    with _lock:
+        if _gspc is None:
+            build()
+            lib = ctypes.CDLL(_GSPC_LIB)
+            lib.gspc_packed_kernel_elems.restype = ctypes.c_size_t
+            lib.gspc_packed_kernel_elems.argtypes = [ctypes.c_int] * 5
+            lib.gspc_pack_kernels.restype = ctypes.c_int
+            lib.gspc_pack_kernels.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7
+            lib.gspc_forward_f32.restype = ctypes.c_int
+            lib.gspc_forward_f32.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 14 + [
+                ctypes.POINTER(ctypes.c_double)]
+            _gspc = lib
+    return _gspc
+
+
+def gspc_pack_kernels(w: np.ndarray, groups: int, T_I: int, T_O: int) -> np.ndarray:
+    """Stage 1 of Algorithm 1 (kernel reshaping; done ahead of time): w [C_out, CPG, KH, KW] -> the 7-D volume
+    [g, KPG/T_O, CPG/T_I, KH, KW, T_I, T_O], returned flat."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    C_out, Cg, KH, KW = w.shape
+    wp = np.empty(w.size, dtype=np.float32)
+    rc = _load_gspc().gspc_pack_kernels(w.ctypes.data, wp.ctypes.data, Cg * groups, C_out, KH, KW, groups, T_I, T_O)
+    if rc != 0:
+        raise ValueError("tile sizes must divide CPG and KPG (Eq. (1) bounds them by CPG and KPG)")
+    return wp
+
+
+def gspc_forward(x: np.ndarray, wp: np.ndarray, w_shape, stride: int, pad: int, dilation: int, groups: int, T_I: int, T_O: int,
+                 threads: int = 1, return_stage_seconds: bool = False):
+    """Stages 2-4 of Algorithm 1 in float32 on kernels packed by gspc_pack_kernels with the same tiles."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    N, C_in, H, W = x.shape
+    C_out, Cg, KH, KW = w_shape
+    Ho = out_dim(H, KH, stride, pad, dilation)
+    Wo = out_dim(W, KW, stride, pad, dilation)
+    y = np.empty((N, C_out, Ho, Wo), dtype=np.float32)
+    secs = (ctypes.c_double * 3)()
+    rc = _load_gspc().gspc_forward_f32(x.ctypes.data, wp.ctypes.data, y.ctypes.data, N, C_in, H, W, C_out, KH, KW, stride, pad,
+                                       dilation, groups, T_I, T_O, int(threads), secs)
+    if rc != 0:
+        raise ValueError("gspc_forward_f32 rejected the problem (%d)" % rc)
+    return (y, tuple(secs)) if return_stage_seconds else y

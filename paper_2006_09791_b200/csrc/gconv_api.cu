@@ -1,4 +1,5 @@
 // Host side of libgconv: descriptor, validation, variant selection and the C ABI of include/gconv.h.
+#include <atomic>
 #include <new>
 
 #include "gconv_internal.h"
@@ -20,8 +21,17 @@ bool variant_supported(const Shape& s, int v) {
     }
 }
 
-// Variant selector.  Keyed on (Cg, Kg, H*W, N) like the tile-size choice the paper leaves to
-// autotuning (Section III-C); the thresholds come from measured timings of the forced variants.
+// Counts weight-packing calls of the whole process.  The tensor-core kernel reads packed weights before its
+// programmatic dependency wait, which is only safe once the packing kernel is known to have completed: a descriptor
+// whose last forward saw an older count launches its next forward as an ordinary (fully serialized) kernel.
+std::atomic<unsigned long long> g_pack_epoch{1};
+
+// Variant selector.  The paper leaves the per-layer choice (its tile sizes) to autotuning (Section III-C); here the
+// measured timings of the forced variants reduce to a rule on the group width alone: the tensor-core variant wherever
+// it supports the shape and a group has at least two channels (narrower groups are merged into block-diagonal ones),
+// the FP32 stream/tiled kernels for depthwise and for 3x3 shapes it rejects, the generic kernel for the rest.  The
+// choices that do depend on (Cg, Kg, H*W, N) -- tiling, filter tile, resident or streamed weights, launch shape --
+// are made inside the tensor-core variant's configuration.
 int select_variant(const Shape& s) {
     if (igemm_supported(s) && s.Cg >= 2) return GCONV_VARIANT_IGEMM_TF32;
     if (tiled_supported(s)) return GCONV_VARIANT_DIRECT_TILED;
@@ -43,11 +53,6 @@ int ensure_device_state(gconv_desc* d) {
         cudaFree(d->status_dev);
         d->status_dev = nullptr;
     }
-    if (d->scratch != nullptr) {
-        cudaFree(d->scratch);
-        d->scratch = nullptr;
-        d->scratch_bytes = 0;
-    }
     e = cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return fail_cuda(d, e);
     e = cudaMalloc(&d->status_dev, sizeof(Status));
@@ -59,6 +64,16 @@ int ensure_device_state(gconv_desc* d) {
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+IgemmLaunchOpts launch_opts(gconv_desc* d) {
+    IgemmLaunchOpts o;
+    const unsigned long long epoch = g_pack_epoch.load(std::memory_order_relaxed);
+    o.pdl = d->pack_epoch_seen == epoch;
+    d->pack_epoch_seen = epoch;
+    o.wait_us = (uint32_t)d->wait_us;
+    o.dbg_skip = d->dbg_skip;
+    return o;
+}
 
 }  // namespace
 
@@ -94,8 +109,11 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
     d->device = -1;
     d->sm_count = 0;
     d->last_cuda_error = 0;
-    d->scratch = nullptr;
-    d->scratch_bytes = 0;
+    d->workspace = nullptr;
+    d->workspace_bytes = 0;
+    d->pack_epoch_seen = 0;
+    d->wait_us = 0;
+    d->dbg_skip = -1;
     *out = d;
     return GCONV_OK;
 }
@@ -103,7 +121,6 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
 int gconv_desc_destroy(gconv_desc_t d) {
     if (d == nullptr) return GCONV_OK;
     if (d->status_dev != nullptr) cudaFree(d->status_dev);
-    if (d->scratch != nullptr) cudaFree(d->scratch);
     delete d;
     return GCONV_OK;
 }
@@ -162,6 +179,7 @@ int gconv_pack_weights(gconv_desc_t d, const float* w_ochw, void* w_packed, void
     if (rc != GCONV_OK) return rc;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e;
+    g_pack_epoch.fetch_add(1, std::memory_order_relaxed);
     switch (d->variant) {
         case GCONV_VARIANT_DIRECT_TILED:
             e = tiled_pack(d->s, w_ochw, w_packed, st);
@@ -190,15 +208,8 @@ int gconv_forward(gconv_desc_t d, const float* x, const void* w_packed, float* y
             break;
         case GCONV_VARIANT_IGEMM_TF32: {
             const size_t need = igemm_scratch_bytes(d->s);
-            if (need > d->scratch_bytes) {   // first forward of a layer that runs on a padded copy of x
-                if (d->scratch != nullptr) cudaFree(d->scratch);
-                d->scratch = nullptr;
-                d->scratch_bytes = 0;
-                e = cudaMalloc(&d->scratch, need);
-                if (e != cudaSuccess) return fail_cuda(d, e);
-                d->scratch_bytes = need;
-            }
-            e = igemm_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st, d->scratch);
+            if (need > 0 && (d->workspace == nullptr || d->workspace_bytes < need)) return GCONV_ERR_WORKSPACE;
+            e = igemm_forward(d->s, x, w_packed, y, d->status_dev, d->sm_count, st, need > 0 ? d->workspace : nullptr, launch_opts(d));
             break;
         }
         case GCONV_VARIANT_DIRECT_GENERIC:
@@ -238,6 +249,7 @@ int gconv_block_pack_weights(gconv_desc_t d, int C2, const float* w_ochw, const 
     if (!igemm_block_supported(d->s, C2)) return GCONV_ERR_UNSUPPORTED;
     int rc = ensure_device_state(d);
     if (rc != GCONV_OK) return rc;
+    g_pack_epoch.fetch_add(1, std::memory_order_relaxed);
     const cudaError_t e = igemm_block_pack(d->s, C2, w_ochw, w2, w_packed, reinterpret_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? GCONV_OK : fail_cuda(d, e);
 }
@@ -248,8 +260,29 @@ int gconv_block_forward(gconv_desc_t d, int C2, const float* x, const void* w_pa
     if (!igemm_block_supported(d->s, C2)) return GCONV_ERR_UNSUPPORTED;
     int rc = ensure_device_state(d);
     if (rc != GCONV_OK) return rc;
-    const cudaError_t e = igemm_block_forward(d->s, C2, x, w_packed, y2, d->status_dev, d->sm_count, reinterpret_cast<cudaStream_t>(stream));
+    const cudaError_t e = igemm_block_forward(d->s, C2, x, w_packed, y2, d->status_dev, d->sm_count, reinterpret_cast<cudaStream_t>(stream),
+                                              launch_opts(d));
     return e == cudaSuccess ? GCONV_OK : fail_cuda(d, e);
+}
+
+size_t gconv_workspace_bytes(gconv_desc_t d) {
+    if (d == nullptr) return 0;
+    return d->variant == GCONV_VARIANT_IGEMM_TF32 ? igemm_scratch_bytes(d->s) : 0;
+}
+
+int gconv_desc_set_workspace(gconv_desc_t d, void* workspace, size_t bytes) {
+    if (d == nullptr) return GCONV_ERR_NULL;
+    if (workspace != nullptr && !aligned16(workspace)) return GCONV_ERR_ALIGNMENT;
+    d->workspace = static_cast<float*>(workspace);
+    d->workspace_bytes = workspace != nullptr ? bytes : 0;
+    return GCONV_OK;
+}
+
+int gconv_desc_set_debug(gconv_desc_t d, int wait_limit_us, int skip_stage) {
+    if (d == nullptr) return GCONV_ERR_NULL;
+    d->wait_us = wait_limit_us > 0 ? wait_limit_us : 0;
+    d->dbg_skip = skip_stage >= 0 ? skip_stage : -1;
+    return GCONV_OK;
 }
 
 int gconv_forward_launches(gconv_desc_t d) {
@@ -284,7 +317,8 @@ const char* gconv_status_string(int status) {
         case GCONV_ERR_CUDA: return "CUDA call failed";
         case GCONV_ERR_PACK_MISMATCH: return "packed weights do not match the descriptor";
         case GCONV_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
-        case GCONV_ERR_TOO_LARGE: return "layer larger than the static scratch (x and y must fit in 16 MiB)";
+        case GCONV_ERR_TOO_LARGE: return "layer larger than the static scratch (x, y and the workspace must fit in 16 MiB)";
+        case GCONV_ERR_WORKSPACE: return "the layer needs a workspace (gconv_workspace_bytes) and none large enough is attached";
         default: return "unknown status";
     }
 }

@@ -23,8 +23,11 @@ struct gconv_desc {
     int device;                  // device the status block lives on (-1 = none yet)
     int sm_count;
     int last_cuda_error;
-    float* scratch;              // lazily allocated device scratch (padded input copy), nullptr for most shapes
-    size_t scratch_bytes;
+    float* workspace;            // caller-owned device workspace attached by gconv_desc_set_workspace (nullptr = none)
+    size_t workspace_bytes;
+    unsigned long long pack_epoch_seen;   // value of the process-wide pack counter at this descriptor's last forward
+    int wait_us;                 // time limit of one bounded wait inside a kernel, microseconds (0 = the default, one second)
+    int dbg_skip;                // failure-path test hook: stage fill that CTA 0's producer leaves out (-1 = none)
 };
 
 namespace gconv {
@@ -145,6 +148,14 @@ struct IgemmCfg {
     FastDiv div_mt, div_spi, div_w;   // tile -> (group/filter tile, pixel tile); pixel tile -> (image, segment or row block); pixel -> (row, column)
     uint32_t stage_bytes;
     size_t smem_bytes;
+    uint32_t wait_us;        // time limit of one bounded wait, microseconds
+    int dbg_skip;            // failure-path test hook: the stage fill CTA 0's producer leaves out (-1 = none)
+};
+// Per-launch options of the tensor-core variant.
+struct IgemmLaunchOpts {
+    bool pdl;                // launch with programmatic stream serialization (set-up overlaps the previous kernel's tail)
+    uint32_t wait_us;        // 0 = default
+    int dbg_skip;            // -1 = none
 };
 bool igemm_supported(const Shape& s);
 IgemmCfg igemm_config(const Shape& s, int sm_count);
@@ -155,9 +166,9 @@ bool igemm_block_supported(const Shape& s, int C2);
 size_t igemm_block_packed_bytes(const Shape& s, int C2);
 cudaError_t igemm_block_pack(const Shape& s, int C2, const float* w, const float* w2, void* packed, cudaStream_t st);
 cudaError_t igemm_block_forward(const Shape& s, int C2, const float* x, const void* packed, float* y2, Status* status, int sm_count,
-                                cudaStream_t st);
-size_t igemm_scratch_bytes(const Shape& s);   // device scratch the forward needs (padded copy of x), 0 for most shapes
+                                cudaStream_t st, const IgemmLaunchOpts& opts);
+size_t igemm_scratch_bytes(const Shape& s);   // device workspace the forward needs (padded copy of x), 0 for most shapes
 cudaError_t igemm_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
-                          cudaStream_t st, float* scratch);
+                          cudaStream_t st, float* scratch, const IgemmLaunchOpts& opts);
 
 }  // namespace gconv

@@ -56,7 +56,7 @@ constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), 
 // Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
 constexpr int kLayoutSMs = 148;
 constexpr uint32_t kPrefetchUses = 1;   // stages whose input is prefetched into L2 before the dependency wait
-constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kDefaultWaitUs = 1000000u;   // a wait gives up after one second unless the descriptor says otherwise
 constexpr int kMaxDynSmem = 226 * 1024;   // 227 KB per CTA minus the static control block (under 1 KB)
 
 struct __align__(8) SharedCtl {
@@ -71,8 +71,10 @@ struct __align__(8) SharedCtl {
     // epilogue group) into a second MMA that accumulates the pointwise output of the pixel tile over all groups (d2)
     unsigned long long a2_full[2], a2_free[2], d2_full[2], d2_free[2], w2_full;
     uint32_t tmem_base;
-    int abort_flag;
+    int abort_flag;      // set by the first role whose wait ran out; every other role then leaves at its next wait
+    uint32_t wait_us;    // time limit of one wait, in microseconds (read as abort_flag[1] by the wait helpers)
 };
+static_assert(offsetof(SharedCtl, wait_us) == offsetof(SharedCtl, abort_flag) + sizeof(int), "wait helpers read the limit behind the flag");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -110,17 +112,40 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
     return ok;
 }
 
-// Bounded wait.  Returns false if the wait ran out or another role already gave up.
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up after the CTA's time limit (one second by default).  Returns false if the wait ran out or
+// another role already gave up; the first role to run out records GCONV_ERR_TIMEOUT with `where` as the detail.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, Status* status,
                                           int where) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t limit_ns = 1000ull * (uint64_t)(uint32_t)abort_flag[1];
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
+        if (global_ns() - t0 > limit_ns) break;
         if (it > 4096) __nanosleep(64);
     }
     *abort_flag = 1;
     record_status(status, GCONV_ERR_TIMEOUT, where);
     return false;
+}
+
+// Drain wait, used only after a role gave up: waits (same time limit) for a phase whose copies may still be in flight.
+// Returns false if it ran out as well.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const uint64_t limit_ns = 1000ull * (uint64_t)(uint32_t)abort_flag[1];
+    const uint64_t t0 = global_ns();
+    while (!mbar_test_wait(bar, parity)) {
+        if (global_ns() - t0 > limit_ns) return false;
+        __nanosleep(64);
+    }
+    return true;
 }
 
 // The same wait for a converged warp: every lane gets the same answer, so the warp never splits
@@ -285,9 +310,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 
     // Programmatic dependent launch: let the next kernel in the stream be scheduled as SMs free up, and run this
     // kernel's own set-up (barriers, TMEM) while the previous kernel drains.  Before griddepcontrol.wait has
-    // returned (the previous kernel's writes complete and visible) the only global memory read is the tag of the
-    // packed weights: they are written by the packing kernel, which never releases its dependents early, so it
-    // had completed before any later kernel of the stream started.
+    // returned (the previous kernel's writes complete and visible) the only global memory read is the packed weights
+    // (their tag here, the first resident bank in the producer).  Only the dependency wait guarantees that an earlier
+    // kernel's writes are visible, so the host launches the first forward after ANY weight packing of the process
+    // without programmatic serialization (a full stream dependency); by every later launch the weights are older than
+    // a completed kernel boundary.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t tag_seen = __ldg(packed);
     const uint8_t* __restrict__ wblocks = reinterpret_cast<const uint8_t*>(packed) + kHeaderBytes;
@@ -318,6 +345,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
         } else if (t == 18) {
             ctl.abort_flag = 0;
+            ctl.wait_us = c.wait_us;
         } else if (c.fuse && t >= 20 && t < 22) {
             mbar_init(smem_u32(&ctl.a2_full[t - 20]), kEpiWarps);
             mbar_init(smem_u32(&ctl.a2_free[t - 20]), 1);
@@ -492,9 +520,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
                 const uint32_t nb = c.b_res ? 0u : (uint32_t)c.nr * blk_bytes;
                 const int chan = g * c.Cg + ch * c.CK;
+                // Failure-path test hook (gconv_desc_set_debug): CTA 0 leaves out one stage fill entirely -- no copy is
+                // issued and the barrier is not armed -- so the consumer's bounded wait on that stage runs out.
+                const bool skip_fill = !pf && (int)it == c.dbg_skip && blockIdx.x == 0;
                 const int lo = tile_f0 + (r - 1) * rstep - c.wseg * 32;
                 const bool box = c.rowbox || c.fast4 == 2 || (c.fast4 == 1 && lo >= 0 && lo + c.nseg * 32 <= HW);
-                if (lane == 0 && pf) {
+                if (skip_fill) {
+                    // nothing
+                } else if (lane == 0 && pf) {
                     if (box) {
                         if (c.rowbox) tma_prefetch_5d(&xmap4, 0, chan, rb_seg, rb_row0, tile_n);
                         else if (c.fast4 == 2) tma_prefetch_4d(&xmap4, 0, chan, lo >> 5, tile_n);
@@ -512,7 +545,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     }
                     if (nb) bulk_load_1d(a_dst + a_all, wtile + (size_t)ks * nb, nb, full);
                 }
-                if (!box) {
+                if (!box && !skip_fill) {
                     if (!have_lane_coords) {
                         uint32_t n, i;
                         if (c.tapb) {                      // lane = 4 * tap + segment: the tap's own row shift, any image
@@ -570,19 +603,19 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         }
         }
         if (!ok && lane == 0) {
-            // drain: wait (bounded) for the copies of every stage that may still be in flight
+            // drain: wait (bounded) for the copies of every stage that may still be in flight, so that no bulk copy
+            // lands in this CTA's shared memory after it has exited; a drain that runs out too is recorded in the
+            // status detail (1000 + stage, 1100 + weight buffer) beside the code of the wait that gave up first
             for (int i = 0; i < c.stages && i < (int)it; ++i) {
                 const uint32_t j = it - 1 - i;
-                const uint32_t bar = smem_u32(&ctl.full[j % c.stages]);
-                for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
-                    if (mbar_try_wait(bar, (j / c.stages) & 1)) break;
+                if ((int)j == c.dbg_skip && blockIdx.x == 0) continue;   // the test hook issued nothing for this fill
+                if (!mbar_drain(smem_u32(&ctl.full[j % c.stages]), (j / c.stages) & 1, abort_flag)) status->detail = 1000 + (int)(j % c.stages);
             }
             for (uint32_t i = 0; i < (uint32_t)c.b_res && i < switches; ++i) {
                 const uint32_t j = switches - 1 - i;
-                const uint32_t bar = smem_u32(&ctl.b_full[c.b_res == 2 ? (j & 1) : 0u]);
+                const uint32_t bb = c.b_res == 2 ? (j & 1) : 0u;
                 const uint32_t par = (c.b_res == 2 ? (j >> 1) : j) & 1;
-                for (uint32_t spin = 0; spin < kSpinLimit; ++spin)
-                    if (mbar_try_wait(bar, par)) break;
+                if (!mbar_drain(smem_u32(&ctl.b_full[bb]), par, abort_flag)) status->detail = 1100 + (int)bb;
             }
         }
     } else if (c.fuse && warp == (c.egroups == 2 ? kMmaWarp3 : kMmaWarp2)) {
@@ -1255,6 +1288,8 @@ size_t igemm_scratch_bytes(const Shape& s_any) {
 static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     const Shape s_true = as_3x3(s_any);
     IgemmCfg c;
+    c.wait_us = kDefaultWaitUs;
+    c.dbg_skip = -1;
     // Pointwise: one vertical tap (a third of the stages and MMAs), one accumulator per filter (N = Kt), filter tiles of
     // up to 128.  Stride 2 computes every pixel and stores the even ones (no stride-2 row tiles: those are built around
     // nine staged rows).
@@ -1280,7 +1315,7 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     if (c.pw) {
         // small planes: narrower filter tiles until there is a tile per SM (each re-reads its pixels from L2)
         const long long px_tiles = ((long long)s.N * s.H * s.W + 127) / 128;
-        while (kt >= 64 && kt % 16 == 0 && (long long)c.groups * (c.Kg / kt) * px_tiles < (long long)sm_count) kt /= 2;
+        while (kt >= 64 && kt % 16 == 0 && (long long)c.groups * (c.Kg / kt) * px_tiles < (long long)kLayoutSMs) kt /= 2;
     }
     c.Kt = kt;
     c.NT = c.Kg / kt;
@@ -1559,13 +1594,23 @@ __global__ void block_pack_w2_kernel(int groups, int Kt, int C2, int C_mid, cons
 }
 }  // namespace
 
-static uint32_t block_tag(const Shape& s, int C2) { return pack_tag(s, GCONV_VARIANT_IGEMM_TF32) ^ (0xB10C0000u + (uint32_t)C2); }
+// Tag of a packed blob of this variant: the shape tag extended by every configuration field the packed layout depends
+// on.  Merge width, filter tile and stage width follow the stride, the batch and the plane size, so weights packed
+// under a descriptor of another batch, plane or stride either have the same layout (and are accepted) or another tag
+// (and the kernel reports GCONV_ERR_PACK_MISMATCH); they are never read in the wrong layout.
+static uint32_t igemm_tag(const Shape& s, const IgemmCfg& c) {
+    uint32_t h = pack_tag(s, GCONV_VARIANT_IGEMM_TF32);
+    const int v[10] = {c.merge, c.groups, c.Cg, c.Kg, c.CK, c.chunks, c.Kt, c.NT, c.Np, c.pw};
+    for (int i = 0; i < 10; ++i) h ^= (uint32_t)v[i] + 0x9e3779b9u + (h << 6) + (h >> 2);
+    return h;
+}
+static uint32_t block_tag(const Shape& s, const IgemmCfg& c, int C2) { return igemm_tag(s, c) ^ (0xB10C0000u + (uint32_t)C2); }
 
 cudaError_t igemm_block_pack(const Shape& s, int C2, const float* w, const float* w2, void* packed, cudaStream_t st) {
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
     const size_t total = (size_t)c.groups * c.NT * 3 * c.chunks * c.Np * c.CK;
     int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
-    igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), block_tag(s, C2));
+    igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), block_tag(s, c, C2));
     const size_t t2 = (size_t)c.groups * c.Kt * C2;
     blocks = (int)((t2 + 255) / 256 < 2368 ? (t2 + 255) / 256 : 2368);
     block_pack_w2_kernel<<<blocks, 256, 0, st>>>(c.groups, c.Kt, C2, s.C_out, w2,
@@ -1582,26 +1627,28 @@ cudaError_t igemm_pack(const Shape& s, const float* w, void* packed, cudaStream_
     const IgemmCfg c = igemm_config(s, 148);
     const size_t total = (size_t)c.groups * c.NT * (c.pw ? 1 : 3) * c.chunks * c.Np * c.CK;
     int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
-    igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), pack_tag(s, GCONV_VARIANT_IGEMM_TF32));
+    igemm_pack_kernel<<<blocks, 256, 0, st>>>(s, c, w, reinterpret_cast<uint32_t*>(packed), igemm_tag(s, c));
     return cudaGetLastError();
 }
 
 static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, const void* packed, float* y, Status* status,
-                                int sm_count, cudaStream_t st, float* scratch);
+                                int sm_count, cudaStream_t st, float* scratch, const IgemmLaunchOpts& opts);
 
 cudaError_t igemm_forward(const Shape& s_true, const float* x_in, const void* packed, float* y, Status* status, int sm_count,
-                          cudaStream_t st, float* scratch) {
-    return igemm_launch(s_true, 0, x_in, packed, y, status, sm_count, st, scratch);
+                          cudaStream_t st, float* scratch, const IgemmLaunchOpts& opts) {
+    return igemm_launch(s_true, 0, x_in, packed, y, status, sm_count, st, scratch, opts);
 }
 
 cudaError_t igemm_block_forward(const Shape& s, int C2, const float* x, const void* packed, float* y2, Status* status, int sm_count,
-                                cudaStream_t st) {
-    return igemm_launch(s, C2, x, packed, y2, status, sm_count, st, nullptr);
+                                cudaStream_t st, const IgemmLaunchOpts& opts) {
+    return igemm_launch(s, C2, x, packed, y2, status, sm_count, st, nullptr, opts);
 }
 
 static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, const void* packed, float* y, Status* status,
-                                int sm_count, cudaStream_t st, float* scratch) {
-    const IgemmCfg c = igemm_config_c2(s_true, sm_count, C2);
+                                int sm_count, cudaStream_t st, float* scratch, const IgemmLaunchOpts& opts) {
+    IgemmCfg c = igemm_config_c2(s_true, sm_count, C2);
+    if (opts.wait_us > 0) c.wait_us = opts.wait_us;
+    c.dbg_skip = opts.dbg_skip;
     Shape s = as_3x3(s_true);
     const float* x = x_in;
     if (c.padded) {
@@ -1715,9 +1762,12 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = 1;
+    // Without the attribute the kernel starts only after everything before it in the stream has completed and is
+    // visible (griddepcontrol.* are then no-ops): used for the first forward after any weight packing, because the
+    // kernel reads the packed weights before its dependency wait.
+    lc.numAttrs = opts.pdl ? 1 : 0;
     return cudaLaunchKernelEx(&lc, kernels[fam], xmap, xmap4, s, cfg, reinterpret_cast<const uint32_t*>(packed), y, status,
-                              C2 > 0 ? block_tag(s_true, C2) : pack_tag(s_true, GCONV_VARIANT_IGEMM_TF32), x);
+                              C2 > 0 ? block_tag(s_true, c, C2) : igemm_tag(s_true, c), x);
 }
 
 

@@ -22,6 +22,7 @@ GCONV_ERR_CUDA = 5
 GCONV_ERR_PACK_MISMATCH = 6
 GCONV_ERR_TIMEOUT = 7
 GCONV_ERR_TOO_LARGE = 8
+GCONV_ERR_WORKSPACE = 9
 
 GCONV_VARIANT_AUTO = 0
 GCONV_VARIANT_DIRECT_GENERIC = 1
@@ -51,6 +52,9 @@ _SIGNATURES = {
     "gconv_block_pack_weights": (ctypes.c_int, [_vp, ctypes.c_int, _vp, _vp, _vp, _vp]),
     "gconv_block_forward": (ctypes.c_int, [_vp, ctypes.c_int, _vp, _vp, _vp, _vp]),
     "gconv_forward_launches": (ctypes.c_int, [_vp]),
+    "gconv_workspace_bytes": (ctypes.c_size_t, [_vp]),
+    "gconv_desc_set_workspace": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t]),
+    "gconv_desc_set_debug": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
     "gconv_last_status": (ctypes.c_int, [_vp, _vp]),
     "gconv_last_cuda_error": (ctypes.c_int, [_vp]),
     "gconv_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -164,7 +168,7 @@ def gconv_forward_host(desc, x_host, w_packed, y_host, x_stage, y_stage, stream=
 
 
 def gconv_forward_host_static(desc, x_host, w_packed, y_host, stream=None) -> None:
-    """Host-buffer forward that allocates nothing (static device scratch, at most 16 MiB of x + y);
+    """Host-buffer forward that allocates nothing (static device scratch, at most 16 MiB of x + y + workspace);
     blocks until y_host is complete and raises on any status other than GCONV_OK."""
     _check(load().gconv_forward_host_static(desc, _ptr(x_host), _ptr(w_packed), _ptr(y_host), _stream(stream)),
            "gconv_forward_host_static")
@@ -192,6 +196,19 @@ def gconv_block_forward(desc, C2: int, x_nchw, w_packed, y2_nchw, stream=None) -
 
 def gconv_forward_launches(desc) -> int:
     return int(load().gconv_forward_launches(desc))
+
+
+def gconv_workspace_bytes(desc) -> int:
+    return int(load().gconv_workspace_bytes(desc))
+
+
+def gconv_desc_set_workspace(desc, workspace, nbytes: int) -> None:
+    """Attach a caller-owned device workspace of `nbytes` bytes (None detaches)."""
+    _check(load().gconv_desc_set_workspace(desc, _ptr(workspace), int(nbytes)), "gconv_desc_set_workspace")
+
+
+def gconv_desc_set_debug(desc, wait_limit_us: int = 0, skip_stage: int = -1) -> None:
+    _check(load().gconv_desc_set_debug(desc, int(wait_limit_us), int(skip_stage)), "gconv_desc_set_debug")
 
 
 def gconv_last_status(desc, stream=None) -> int:

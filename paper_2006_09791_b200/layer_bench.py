@@ -19,6 +19,7 @@ import torch
 
 from . import build as gbuild
 from . import gconv, synth
+from .torch_util import attach_workspace
 from .workloads import Layer
 
 VARIANTS = {"auto": gconv.GCONV_VARIANT_AUTO, "generic": gconv.GCONV_VARIANT_DIRECT_GENERIC,
@@ -53,6 +54,7 @@ def main():
     d = gconv.gconv_desc_create(*L.desc_args())
     if VARIANTS[a.variant]:
         gconv.gconv_desc_set_variant(d, VARIANTS[a.variant])
+    ws = attach_workspace(d, dev)
     s = torch.cuda.Stream()
     torch.cuda.synchronize()
     if a.c2:

@@ -15,6 +15,7 @@ import torch
 
 from . import build as gbuild
 from . import gconv, synth
+from .torch_util import attach_workspace
 from .workloads import Layer, resnet34_layers, resnext_layers, sweep_layers, wrn_stack
 
 VARIANTS = [(gconv.GCONV_VARIANT_DIRECT_GENERIC, "generic"), (gconv.GCONV_VARIANT_DIRECT_TILED, "tiled"),
@@ -28,6 +29,7 @@ def time_variant(L, variant, reps=20):
         if not gconv.gconv_variant_supported(d, variant):
             return None
         gconv.gconv_desc_set_variant(d, variant)
+        ws = attach_workspace(d, dev)
         per = 4 * (L.x_elems + L.y_elems)
         nbuf = max(2, min(64, -(-(2 * 126 * 2 ** 20 + (64 << 20)) // per)))
         x0, w0 = synth.make_layer_tensors(min(L.N, 2), L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 5, L.x_dist)

@@ -4,6 +4,7 @@ import torch
 
 import oracle
 from paper_2006_09791_b200 import gconv, synth
+from paper_2006_09791_b200.torch_util import attach_workspace
 
 
 def run_layer(L, x_np, w_np, variant=gconv.GCONV_VARIANT_AUTO, stream=None, guard=64):
@@ -15,6 +16,7 @@ def run_layer(L, x_np, w_np, variant=gconv.GCONV_VARIANT_AUTO, stream=None, guar
         if variant != gconv.GCONV_VARIANT_AUTO:
             gconv.gconv_desc_set_variant(d, variant)
         used = gconv.gconv_variant(d)
+        ws = attach_workspace(d, dev)    # None for most layers
         x = torch.from_numpy(x_np).to(dev)
         w = torch.from_numpy(w_np).to(dev)
         pb = gconv.gconv_packed_bytes(d)

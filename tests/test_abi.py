@@ -7,7 +7,8 @@ import pytest
 
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv
-from paper_2006_09791_b200.workloads import Layer, config0, resnet34_layers, wrn_stack
+from paper_2006_09791_b200.workloads import (R34_GROUPS, Layer, config0, mobilenetv2_dw_layers, resnet34_layers, resnext_layers, sweep_layers,
+                                             wrn_stack)
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -76,3 +77,39 @@ def test_null_and_variant_errors():
     finally:
         gconv.gconv_desc_destroy(d)
     assert gconv.status_string(gconv.GCONV_ERR_TIMEOUT) and gconv.variant_name(3) == "igemm_tf32"
+
+
+def test_workspace_is_caller_owned_and_rarely_needed():
+    """gconv_forward allocates nothing: the few layers that compute on a zero-padded copy of x report the bytes they
+    need and refuse to run without an attached workspace; layers whose width is a multiple of 4 never need one."""
+    lib = gconv.load()
+    assert lib.gconv_workspace_bytes(None) == 0
+    bench_layers = config0() + wrn_stack(1, 128) + wrn_stack(16, 128) + sweep_layers(32) + resnext_layers(64) + mobilenetv2_dw_layers(64)
+    for g in R34_GROUPS:
+        bench_layers += resnet34_layers(g, 64)
+    for L in bench_layers:
+        d = gconv.gconv_desc_create(*L.desc_args())
+        try:
+            need = gconv.gconv_workspace_bytes(d)
+            assert need == 0 or L.W % 4 != 0, (L.name, L.groups)
+            assert gconv.gconv_forward_launches(d) == (2 if need else 1), (L.name, L.groups)
+        finally:
+            gconv.gconv_desc_destroy(d)
+    # a width the bulk tensor copies cannot address, with groups too wide for the copy-warp path: padded copy of x
+    L = Layer("w18", 4, 128, 18, 18, 128, groups=1)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        if gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32 and gconv.gconv_workspace_bytes(d) > 0:
+            assert gconv.gconv_workspace_bytes(d) == 4 * L.N * L.C_in * 18 * 20       # rows padded from 18 to 20 columns
+            assert gconv.gconv_forward_launches(d) == 2
+            # no workspace attached: nothing is enqueued (the pointers are never touched), and no device is needed
+            assert lib.gconv_forward(d, 16, 16, 32, None) in (gconv.GCONV_ERR_WORKSPACE, gconv.GCONV_ERR_CUDA)
+            assert lib.gconv_desc_set_workspace(d, 8, 1 << 20) == gconv.GCONV_ERR_ALIGNMENT
+            assert lib.gconv_desc_set_workspace(d, 0, 0) == gconv.GCONV_OK
+        gconv.gconv_desc_set_variant(d, gconv.GCONV_VARIANT_DIRECT_GENERIC)
+        assert gconv.gconv_workspace_bytes(d) == 0
+    finally:
+        gconv.gconv_desc_destroy(d)
+    assert lib.gconv_desc_set_workspace(None, 0, 0) == gconv.GCONV_ERR_NULL
+    assert lib.gconv_desc_set_debug(None, 0, -1) == gconv.GCONV_ERR_NULL
+    assert "workspace" in gconv.status_string(gconv.GCONV_ERR_WORKSPACE)

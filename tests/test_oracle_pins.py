@@ -10,7 +10,6 @@ from paper_2006_09791_b200 import synth
 from paper_2006_09791_b200.workloads import Layer
 
 from golden_io import load_case, load_numbers
-from gspc_alg1 import gspc
 
 GOLDEN_CASES = ["fig3_shape_index_valued.txt", "delta_no_flip.txt", "ones_zero_padding.txt",
                 "stride2_pad1.txt", "dilation2.txt", "two_groups_asymmetric.txt"]
@@ -98,18 +97,62 @@ def test_matches_torch_conv2d_float64(cfg):
     np.testing.assert_allclose(got, want.numpy(), rtol=0, atol=1e-12)
 
 
-def test_gspc_algorithm1_agrees():
-    """The paper's four-stage packed algorithm computes the same tensor for several tile sizes."""
-    N, C_in, C_out, g, H, W, KH, KW, s, p = 2, 8, 12, 2, 6, 5, 3, 2, 2, 1
-    x = _rand((N, C_in, H, W), 31, 0)
-    w = _rand((C_out, C_in // g, KH, KW), 31, 1)
-    want = oracle.gconv_ref(x, w, s, p, 1, g)
-    for T_I, T_O in [(1, 1), (2, 3), (4, 6), (4, 2)]:
-        np.testing.assert_allclose(gspc(x, w, s, p, g, T_I, T_O), want, rtol=0, atol=1e-12)
-    # the Fig. 3 shape with its stated tile sizes T_I = T_O = 2
+def _im2col_matmul(x, w, stride, pad, dilation, groups):
+    """A formulation that shares nothing with the oracle's loop nest: per group, the zero-padded input is unfolded
+    into a [Cg*KH*KW, H_out*W_out] matrix with numpy slicing and multiplied by the [Kg, Cg*KH*KW] filter matrix."""
+    x = np.asarray(x, np.float64)
+    w = np.asarray(w, np.float64)
+    N, C_in, H, W = x.shape
+    C_out, Cg, KH, KW = w.shape
+    Kg = C_out // groups
+    xp = np.pad(x, ((0, 0), (0, 0), (pad, pad), (pad, pad)))
+    Ho = (H + 2 * pad - dilation * (KH - 1) - 1) // stride + 1
+    Wo = (W + 2 * pad - dilation * (KW - 1) - 1) // stride + 1
+    y = np.empty((N, C_out, Ho, Wo))
+    for n in range(N):
+        for g in range(groups):
+            cols = np.stack([xp[n, g * Cg + c, r * dilation:r * dilation + (Ho - 1) * stride + 1:stride,
+                                s * dilation:s * dilation + (Wo - 1) * stride + 1:stride].reshape(-1)
+                             for c in range(Cg) for r in range(KH) for s in range(KW)])
+            y[n, g * Kg:(g + 1) * Kg] = (w[g * Kg:(g + 1) * Kg].reshape(Kg, -1) @ cols).reshape(Kg, Ho, Wo)
+    return y
+
+
+def test_unfold_and_matmul_agrees():
+    """The oracle against the im2col + matrix-product formulation of the same definition (Section II), over strides,
+    paddings, dilations, unequal Cg and Kg and non-square kernels."""
+    for seed, (N, C_in, C_out, g, H, W, KH, KW, s, p, d) in enumerate([
+            (2, 8, 12, 2, 6, 5, 3, 2, 2, 1, 1), (1, 6, 6, 6, 9, 9, 3, 3, 1, 1, 1), (2, 4, 8, 1, 7, 10, 3, 3, 1, 2, 2),
+            (1, 12, 6, 3, 11, 8, 5, 3, 3, 2, 1), (3, 16, 16, 4, 8, 8, 1, 1, 2, 0, 1)]):
+        x = _rand((N, C_in, H, W), 131 + seed, 0)
+        w = _rand((C_out, C_in // g, KH, KW), 131 + seed, 1)
+        np.testing.assert_allclose(oracle.gconv_ref(x, w, s, p, d, g), _im2col_matmul(x, w, s, p, d, g), rtol=0, atol=1e-12)
+
+
+def test_gspc_baseline_is_pinned_to_the_oracle():
+    """The float32 CPU program of the paper's method (Algorithm 1, Section III-B: four stages, tiles T_I and T_O) that
+    the benchmark times as its second CPU baseline computes the oracle's tensor, for tile pairs from (1, 1) up to the
+    bounds of Eq. (1) (T_I = CPG, T_O = KPG); tile sizes that do not divide are rejected."""
+    cases = [(2, 8, 12, 2, 6, 5, 3, 2, 2, 1, 1, [(1, 1), (2, 3), (4, 6), (4, 2)]),
+             (1, 16, 16, 4, 14, 14, 3, 3, 1, 1, 1, [(1, 4), (4, 4), (2, 1)]),
+             (3, 6, 6, 6, 8, 9, 3, 3, 2, 1, 1, [(1, 1)]),                      # depthwise: both tiles can only be 1
+             (1, 32, 64, 1, 9, 9, 3, 3, 1, 2, 2, [(8, 16), (32, 64), (1, 8)])]
+    for seed, (N, C_in, C_out, g, H, W, KH, KW, s, p, d, tiles) in enumerate(cases):
+        x = _rand((N, C_in, H, W), 31 + seed, 0)
+        w = _rand((C_out, C_in // g, KH, KW), 31 + seed, 1)
+        want = oracle.gconv_ref(x, w, s, p, d, g)
+        for T_I, T_O in tiles:
+            wp = oracle.gspc_pack_kernels(w, g, T_I, T_O)
+            for threads in (1, 3):
+                got = oracle.gspc_forward(x, wp, w.shape, s, p, d, g, T_I, T_O, threads=threads)
+                assert np.max(np.abs(got - want)) <= 1e-5 * np.max(np.abs(want)), (seed, T_I, T_O)
+    with pytest.raises(ValueError):
+        oracle.gspc_pack_kernels(np.zeros((12, 4, 3, 3), np.float32), 2, 3, 4)     # T_I = 3 does not divide CPG = 4
+    # the Fig. 3 shape with its stated tile sizes T_I = T_O = 2 (small integers: exact in float32)
     x = np.arange(16, dtype=np.float32).reshape(1, 4, 2, 2)
     w = np.arange(32, dtype=np.float32).reshape(4, 2, 2, 2)
-    np.testing.assert_array_equal(gspc(x, w, 1, 0, 2, 2, 2).ravel(), [140, 364, 1836, 2572])
+    got = oracle.gspc_forward(x, oracle.gspc_pack_kernels(w, 2, 2, 2), w.shape, 1, 0, 1, 2, 2, 2)
+    np.testing.assert_array_equal(got.ravel(), [140, 364, 1836, 2572])
 
 
 def test_mac_counter_closed_form_and_table1():

@@ -8,6 +8,7 @@ import torch
 import oracle
 from paper_2006_09791_b200 import build as gbuild
 from paper_2006_09791_b200 import gconv, synth
+from paper_2006_09791_b200.torch_util import attach_workspace
 from paper_2006_09791_b200.workloads import (Layer, config0, depthwise5x5_layers, mobilenetv2_dw_layers, resnet34_layers, resnext_layers,
                                              sweep_layers, wrn_stack)
 
@@ -242,7 +243,7 @@ def test_wrn_stack_small_batch(groups):
                     check_layer(L, v)
 
 
-@pytest.mark.parametrize("groups", [1, 4, 32])
+@pytest.mark.parametrize("groups", [1, 2, 4, 8, 16, 32])
 def test_resnet34_shapes(groups):
     for L in resnet34_layers(groups, 2):
         check_layer(L)
@@ -336,6 +337,7 @@ def test_dependent_chain_back_to_back(shape):
     try:
         stream = torch.cuda.Stream()
         with torch.cuda.stream(stream):
+            wss = [attach_workspace(d, dev) for d in descs]
             bufs = [torch.from_numpy(x0).to(dev)] + [torch.empty(L.y_elems, dtype=torch.float32, device=dev) for _ in range(depth)]
             wps = []
             for d, w in zip(descs, ws):
@@ -351,10 +353,7 @@ def test_dependent_chain_back_to_back(shape):
                 for b in bufs[1:]:
                     b.fill_(float("nan"))
                 if use_graph:
-                    run_chain()                      # (descriptor-owned allocations happen outside the capture)
                     stream.synchronize()
-                    for b in bufs[1:]:
-                        b.fill_(float("nan"))
                     graph = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(graph, stream=stream):
                         run_chain()
@@ -375,6 +374,77 @@ def test_dependent_chain_back_to_back(shape):
     finally:
         for d in descs:
             gconv.gconv_desc_destroy(d)
+
+
+def _stack_chain(layers, groups, seed, batches_checked):
+    """Runs `layers` as a real chain (layer k reads layer k-1's output) on one stream, eagerly and as a CUDA-graph replay
+    over NaN-filled buffers, and compares every layer's output with the oracle applied to the input that layer saw."""
+    dev = torch.device("cuda:0")
+    L0 = layers[0]
+    x0, _ = synth.make_layer_tensors(L0.N, L0.C_in, L0.H, L0.W, L0.C_out, 3, 3, groups, synth.layer_seed(seed, L0.N, groups))
+    ws = [synth.make_layer_tensors(1, L.C_in, L.H, L.W, L.C_out, 3, 3, groups, synth.layer_seed(seed + 1, k, groups))[1]
+          for k, L in enumerate(layers)]
+    descs = [gconv.gconv_desc_create(*L.desc_args()) for L in layers]
+    try:
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            wss = [attach_workspace(d, dev) for d in descs]
+            bufs = [torch.from_numpy(x0).to(dev)] + [torch.empty(L.y_elems, dtype=torch.float32, device=dev) for L in layers]
+            wps = []
+            for d, w in zip(descs, ws):
+                wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+                gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp, stream)
+                wps.append(wp)
+
+            def run_chain():
+                for k, d in enumerate(descs):
+                    gconv.gconv_forward(d, bufs[k], wps[k], bufs[k + 1], stream)
+
+            for use_graph in batches_checked:
+                for b in bufs[1:]:
+                    b.fill_(float("nan"))
+                if use_graph:
+                    stream.synchronize()
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=stream):
+                        run_chain()
+                    for b in bufs[1:]:
+                        b.fill_(float("nan"))
+                    graph.replay()
+                else:
+                    run_chain()
+                stream.synchronize()
+                for d in descs:
+                    assert gconv.gconv_last_status(d, stream) == gconv.GCONV_OK
+                seen = bufs[0].cpu().numpy().reshape(L0.N, L0.C_in, L0.H, L0.W)
+                for k, L in enumerate(layers):
+                    got = bufs[k + 1].cpu().numpy().reshape(L.N, L.C_out, L.H_out, L.W_out)
+                    assert np.all(np.isfinite(got)), "layer %d (%s) wrote a non-finite value or skipped one" % (k, L.name)
+                    ref = oracle.gconv_ref(seen, ws[k], L.stride, L.pad, L.dilation, groups, threads=oracle.max_threads())
+                    err = rel_err(got, ref)
+                    assert err <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(descs[k])], (k, L.name, use_graph, err)
+                    seen = got
+    finally:
+        for d in descs:
+            gconv.gconv_desc_destroy(d)
+
+
+@pytest.mark.parametrize("groups,N", [(1, 1), (2, 3), (4, 128), (8, 5), (16, 1), (1, 128)])
+def test_wrn_stack_as_a_real_chain(groups, N):
+    """The 18 layers of the WRN-40-2-shaped stack in network order -- six 32-channel layers at 32x32, the stride-2
+    transition to 64 channels, five layers at 16x16, the stride-2 transition to 128 channels, five layers at 8x8 --
+    each reading its predecessor's output.  This is the chain the bench replays at batch 1."""
+    layers = []
+    for L in wrn_stack(groups, N):
+        layers.extend([L] * L.repeat)
+    assert len(layers) == 18 and layers[6].stride == 2 and layers[12].stride == 2
+    _stack_chain(layers, groups, 51, (False, True))
+
+
+@pytest.mark.parametrize("groups,N", [(1, 1), (4, 2), (32, 1)])
+def test_resnet34_stack_as_a_real_chain(groups, N):
+    """The ResNet-34-shaped layers in network order (56x56 down to 7x7 through three stride-2 transitions), chained."""
+    _stack_chain(resnet34_layers(groups, N), groups, 53, (False, True))
 
 
 BLOCK_SHAPES = [
@@ -448,6 +518,109 @@ def test_pack_mismatch_is_reported_not_fatal():
         assert gconv.gconv_last_status(d) == gconv.GCONV_OK
         y_ref = oracle.gconv_ref(x, w, 1, 1, 1, L.groups)
         assert rel_err(y.cpu().numpy().reshape(y_ref.shape), y_ref) <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(d)]
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
+def test_weights_packed_under_another_batch_plane_or_stride():
+    """The tensor-core variant's packed layout follows more than the filter shape (merge width and filter tile depend on
+    the stride, the batch and the plane size).  Weights packed under a descriptor with the same filters but another
+    batch, plane or stride must give either the right y or GCONV_ERR_PACK_MISMATCH with y untouched -- never a wrong y."""
+    dev = torch.device("cuda:0")
+    pairs = [
+        # (descriptor the weights are packed under, descriptor that runs them)
+        (Layer("pw_n1", 1, 128, 8, 8, 128, 1, 1, 1, 0, 1, 1), Layer("pw_n1024", 1024, 128, 8, 8, 128, 1, 1, 1, 0, 1, 1)),
+        (Layer("g8_s1", 4, 64, 32, 32, 128, groups=8), Layer("g8_s2", 4, 64, 32, 32, 128, stride=2, groups=8)),
+        (Layer("wide_n2", 2, 256, 56, 56, 256), Layer("wide_n32", 32, 256, 56, 56, 256)),
+        (Layer("same_a", 2, 32, 32, 32, 32, groups=4), Layer("same_b", 7, 32, 16, 16, 32, groups=4)),
+    ]
+    outcomes = set()
+    for La, Lb in pairs:
+        x, w = synth.make_layer_tensors(Lb.N, Lb.C_in, Lb.H, Lb.W, Lb.C_out, Lb.KH, Lb.KW, Lb.groups, synth.layer_seed(61, Lb.N, Lb.H))
+        da, db = gconv.gconv_desc_create(*La.desc_args()), gconv.gconv_desc_create(*Lb.desc_args())
+        try:
+            assert gconv.gconv_variant(da) == gconv.gconv_variant(db) == gconv.GCONV_VARIANT_IGEMM_TF32
+            nb = max(gconv.gconv_packed_bytes(da), gconv.gconv_packed_bytes(db))
+            wp = torch.zeros(nb // 4, dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(da, torch.from_numpy(w).to(dev), wp)
+            y = torch.full((Lb.y_elems,), 7.0, dtype=torch.float32, device=dev)
+            gconv.gconv_forward(db, torch.from_numpy(x).to(dev), wp, y)
+            st = gconv.gconv_last_status(db)
+            if st == gconv.GCONV_ERR_PACK_MISMATCH:
+                assert bool((y == 7.0).all())
+            else:
+                assert st == gconv.GCONV_OK
+                ref = oracle.gconv_ref(x, w, Lb.stride, Lb.pad, Lb.dilation, Lb.groups, threads=oracle.max_threads())
+                assert rel_err(y.cpu().numpy().reshape(ref.shape), ref) <= gconv.VARIANT_TOLERANCE[gconv.GCONV_VARIANT_IGEMM_TF32]
+            outcomes.add(st)
+        finally:
+            gconv.gconv_desc_destroy(da)
+            gconv.gconv_desc_destroy(db)
+    assert outcomes == {gconv.GCONV_OK, gconv.GCONV_ERR_PACK_MISMATCH}     # both outcomes occur among the pairs
+
+
+def test_bounded_wait_runs_out_and_the_context_survives():
+    """Failure path of the tensor-core kernel.  The test hook makes the first thread block's producer leave out one
+    stage fill (nothing is issued, the barrier is never armed); the consumer's wait on it must give up after the time
+    limit, the kernel must return with GCONV_ERR_TIMEOUT recorded, and the next ordinary forward of the same
+    descriptor must be correct (tensor memory was freed, the context is intact).  Nothing faults, traps or hangs."""
+    dev = torch.device("cuda:0")
+    for L, skip in ((Layer("to_a", 8, 32, 32, 32, 32, groups=4), 0), (Layer("to_b", 6, 128, 28, 28, 128), 3)):
+        x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, synth.layer_seed(63, L.N))
+        d = gconv.gconv_desc_create(*L.desc_args())
+        try:
+            assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32
+            wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+            xd = torch.from_numpy(x).to(dev)
+            y = torch.zeros(L.y_elems, dtype=torch.float32, device=dev)
+            gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
+            gconv.gconv_desc_set_debug(d, wait_limit_us=2000, skip_stage=skip)
+            t0 = torch.cuda.Event(enable_timing=True)
+            t1 = torch.cuda.Event(enable_timing=True)
+            t0.record()
+            gconv.gconv_forward(d, xd, wp, y)
+            t1.record()
+            assert gconv.gconv_last_status(d) == gconv.GCONV_ERR_TIMEOUT
+            assert t0.elapsed_time(t1) < 500.0            # a handful of 2 ms waits, not the default second, not forever
+            assert gconv.gconv_last_status(d) == gconv.GCONV_OK       # reading clears it
+            gconv.gconv_desc_set_debug(d, 0, -1)
+            for _ in range(2):
+                y.fill_(float("nan"))
+                gconv.gconv_forward(d, xd, wp, y)
+                assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+                ref = oracle.gconv_ref(x, w, 1, 1, 1, L.groups, threads=oracle.max_threads())
+                assert rel_err(y.cpu().numpy().reshape(ref.shape), ref) <= gconv.VARIANT_TOLERANCE[gconv.GCONV_VARIANT_IGEMM_TF32]
+        finally:
+            gconv.gconv_desc_destroy(d)
+
+
+def test_padded_copy_layers_need_an_attached_workspace():
+    """Widths the bulk tensor copies cannot address with groups the copy warps do not serve: gconv_forward allocates
+    nothing, it refuses to run until the caller attaches the workspace, then runs in two launches."""
+    dev = torch.device("cuda:0")
+    L = Layer("w18", 3, 128, 18, 18, 128, groups=1)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        need = gconv.gconv_workspace_bytes(d)
+        if need == 0:
+            pytest.skip("this build serves the shape without a workspace")
+        x, w = synth.make_layer_tensors(L.N, L.C_in, L.H, L.W, L.C_out, 3, 3, L.groups, 71)
+        wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+        xd = torch.from_numpy(x).to(dev)
+        y = torch.full((L.y_elems,), 7.0, dtype=torch.float32, device=dev)
+        gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
+        free0 = torch.cuda.mem_get_info()[0]
+        with pytest.raises(gconv.GconvError) as e:
+            gconv.gconv_forward(d, xd, wp, y)
+        assert e.value.status == gconv.GCONV_ERR_WORKSPACE and bool((y == 7.0).all())
+        ws = attach_workspace(d, dev)
+        assert ws is not None and ws.numel() * 4 >= need
+        free1 = torch.cuda.mem_get_info()[0]
+        gconv.gconv_forward(d, xd, wp, y)
+        assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+        assert torch.cuda.mem_get_info()[0] == free1 and free1 <= free0     # the forward itself allocated nothing
+        ref = oracle.gconv_ref(x, w, 1, 1, 1, L.groups, threads=oracle.max_threads())
+        assert rel_err(y.cpu().numpy().reshape(ref.shape), ref) <= gconv.VARIANT_TOLERANCE[gconv.gconv_variant(d)]
     finally:
         gconv.gconv_desc_destroy(d)
 
