@@ -130,7 +130,13 @@ struct IgemmCfg {
     // fused grouped + pointwise block (0 for the plain convolution)
     int fuse, C2, n_gn, d2_col;   // pointwise output channels, (group, filter tile) pairs per pixel tile, TMEM column of its accumulator
     int pw;                       // pointwise layer, stride 1: one vertical tap per chunk, one accumulator per filter (N = Kt)
-    int soft;                     // copy warps stage the input with cp.async (widths TMA cannot address); no padded copy of x
+    int soft;                     // gather producer: raw input rows land in a ring by bulk copy, copy warps build the operand stages from
+                                  // them (1: stride 1, three vertical-tap blocks; 2: stride 2, even/odd column blocks per tap)
+    int rps, IPT;                 // gather tilings: output rows per 32-lane segment; whole images per tile (1: a tile is part of one image)
+    int boxpx, pieces, raw_whole, raw_bulk;   // raw part = `pieces` boxes of boxpx flat pixels x CK channels; parts hold whole planes; one 1-D copy per part
+    int raw_stages;               // depth of the raw ring
+    uint32_t raw_off, raw_bytes;  // shared-memory offset of the raw ring, bytes per raw buffer
+    FastDiv div_boxpx;
     int ball;                     // every (group, filter tile) keeps a resident weight buffer of its own: no switches
     int d2_bufs;                  // pointwise accumulators in TMEM (2 when the columns allow: alternate pixel tiles)
     uint32_t w2_off, a2_off;      // shared-memory offsets of the resident pointwise weights and of the two A2 buffers

@@ -38,6 +38,7 @@
 // wait runs out the kernel records GCONV_ERR_TIMEOUT, all roles leave their loops, outstanding bulk
 // copies are waited for (bounded), TMEM is freed and the kernel returns.
 #include <cuda.h>
+#include <string.h>
 
 #include "gconv_internal.h"
 
@@ -50,7 +51,7 @@ constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the fir
 constexpr int kEpi2First = kMmaWarp2 + 1;    // first warp of the second epilogue group
 constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issuing warps (used when four accumulators fit)
 constexpr int kThreads = 32 * (kMmaWarp3 + 2);
-constexpr int kSoftWarps = 4;        // copy warps of the software producer (light launch shape only): warps kEpi2First ...
+constexpr int kSoftWarps = 4;        // copy warps of the gather producer, one per segment of a tile: warps kEpi2First ... in the light shape
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 // Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
@@ -70,6 +71,7 @@ struct __align__(8) SharedCtl {
     // fused grouped + pointwise block: the grouped result of a tile goes through shared memory (a2, one buffer per
     // epilogue group) into a second MMA that accumulates the pointwise output of the pixel tile over all groups (d2)
     unsigned long long a2_full[2], a2_free[2], d2_full[2], d2_free[2], w2_full;
+    unsigned long long raw_full[4], raw_empty[4];   // gather producer: ring of raw input buffers (bulk copies in, copy warps out)
     uint32_t tmem_base;
     int abort_flag;      // set by the first role whose wait ran out; every other role then leaves at its next wait
     uint32_t wait_us;    // time limit of one wait, in microseconds (read as abort_flag[1] by the wait helpers)
@@ -248,6 +250,41 @@ __device__ __forceinline__ void tile_coords(const IgemmCfg& c, uint32_t tile, ui
     }
 }
 
+// Gather tilings (c.soft).  A segment is `rps` whole output rows side by side in 32 lanes.  With at least three segments
+// per image a tile is four consecutive segments of ONE image (TPI tiles per image, the last one possibly short) and its
+// raw buffer holds one part: the input rows those segments need.  Smaller planes put IPT = 4 / SPI whole images into a
+// tile, one part (whole plane) per image.
+__device__ __forceinline__ void gath_segment(const IgemmCfg& c, uint32_t mt, int wq, int& n, int& i, int& part) {
+    if (c.IPT == 1) {
+        uint32_t nn, t;
+        c.div_spi.divmod(mt, nn, t);              // div_spi divides by the tiles per image
+        n = (int)nn;
+        i = (int)t * 4 + wq;
+        part = 0;
+    } else {
+        part = c.SPI == 2 ? (wq >> 1) : wq;
+        i = c.SPI == 2 ? (wq & 1) : 0;
+        n = (int)mt * c.IPT + part;
+    }
+}
+// Part `part` of tile mt's raw buffer: the image it is read from and the flat pixel (a multiple of 4) it starts at.
+__device__ __forceinline__ void gath_part(const Shape& s, const IgemmCfg& c, uint32_t mt, int part, int& n, int& fa) {
+    fa = 0;
+    if (c.IPT == 1) {
+        uint32_t nn, t;
+        c.div_spi.divmod(mt, nn, t);
+        n = (int)nn;
+        if (!c.raw_whole) {
+            const int p0 = (int)t * 4 * c.rps;    // first output row of the tile
+            int h_lo = c.soft == 2 ? 2 * p0 - 1 : p0 - s.dilation;
+            if (h_lo < 0) h_lo = 0;
+            fa = (h_lo * s.W) & ~3;
+        }
+    } else {
+        n = (int)mt * c.IPT + part;
+    }
+}
+
 // Families: sets of configuration fields fixed at compile time (-1 = left to the run-time configuration).  The kernel
 // body is written once against the run-time configuration; a family instantiation overwrites the listed fields of a
 // local copy with constants, and the compiler drops every path they rule out.  The role code is a single warp (often a
@@ -257,7 +294,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 26;
+constexpr int kFamilies = 28;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -274,8 +311,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1,  0,  0}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
          : f == 13 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  1,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0,  0}     // fused block, 32-wide planes, two CTAs per SM
          : f == 14 ? Family{1,  0,  3,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  1, -1,  0,  0}     // fused block, row boxes, two resident banks
-         : f == 15 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  4,  12,  0,  0,  1,  0,  0,  1,  0}     // copy-warp producer (14x14, 7x7 planes), tap blocks
-         : f == 16 ? Family{0,  1,  1,  0,   1,  1,  0,  1, -1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0,  0,  0,  0,  0,  1,  0}     // copy-warp producer, one stage per tap
+         : f == 15 ? Family{0,  0,  3,  0,   1,  1,  0,  1,  1, 16, -1, -1,  -1, -1,  2,  2,  0,  0,  4,  12,  0, -1,  0,  0,  0,  1,  0}     // gather producer, stride 1 (14x14, 7x7, ... planes), narrow groups, 16-channel stages
+         : f == 16 ? Family{0,  0,  3,  0,   1,  1,  0,  1,  2, 16, -1, -1,  -1, -1,  2,  2,  0,  0,  8,  24,  0, -1,  0,  0,  0,  2,  0}     // gather producer, stride 2 (even/odd column blocks), narrow groups, 16-channel stages
          : f == 17 ? Family{0, 1, 1, 0, 1, 1, 0, 1, -1, 32, -1, -1, -1, -1, 2, 2, 0, 0, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, two CTAs per SM
          : f == 18 ? Family{1, 0, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, -1, 1, 0, 0, 0, 0, 1}     // pointwise, row boxes
          : f == 19 ? Family{0, 1, 1, 0, -1, -1, 0, 1, -1, 32, -1, -1, -1, -1, -1, -1, 0, -1, 0, 4, 0, -1, 0, 0, 0, 0, 1}     // pointwise, segment tilings, one CTA per SM
@@ -285,6 +322,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 23 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 16, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one large resident bank, 16-channel stages
          : f == 24 ? Family{1,   0,  3,  0,   1,  2,  1,  2,  2, 16, -1, 64, 192, -1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, one resident 64-filter bank, 16-channel stages
          : f == 25 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 16, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights, 16-channel stages
+         : f == 26 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  1,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  4,  12,  0, -1,  0,  0,  0,  1,  0,  0}     // gather producer, stride 1, 8-channel stages
+         : f == 27 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  2,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  8,  24,  0, -1,  0,  0,  0,  2,  0,  0}     // gather producer, stride 2, 8-channel stages
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -331,8 +370,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         const int t = (int)threadIdx.x - 64;
         if (t >= 0 && t < 8) {
             if (t < c.stages) {
-                mbar_init(smem_u32(&ctl.full[t]), c.soft ? (uint32_t)kSoftWarps : 1u);
+                mbar_init(smem_u32(&ctl.full[t]), c.soft ? (uint32_t)kSoftWarps + (c.b_res ? 0u : 1u) : 1u);   // copy warps (+ the streamed weights' arm)
                 mbar_init(smem_u32(&ctl.empty[t]), 1);
+            }
+            if (c.soft && t < 4) {
+                mbar_init(smem_u32(&ctl.raw_full[t]), 1);
+                mbar_init(smem_u32(&ctl.raw_empty[t]), kSoftWarps);
             }
         } else if (t >= 8 && t < 8 + kMaxAcc) {
             const int i = t - 8;
@@ -470,7 +513,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const uint8_t* wtile = wblocks + (size_t)gn * b_tile_bytes;
             const bool switch_b = !pf && c.b_res && !c.ball && (int)gn != cur_gn;
             if (c.soft) {
-                // the copy warps stage the input; this warp only brings the resident weights of a new (group, filter tile)
+                // Gather producer: this warp brings the resident weights of a new (group, filter tile) and, per stage, the
+                // raw input of the tile's parts into the raw ring (tiled boxes of flat pixels x channels, or one bulk copy
+                // of whole planes where the plane is not a multiple of 16 bytes) plus -- with streamed weights -- the
+                // stage's weight blocks.  The copy warps turn raw buffers into operand stages.
                 if (switch_b) {
                     const uint32_t bb = c.b_res == 2 ? (switches & 1) : 0u, use = c.b_res == 2 ? (switches >> 1) : switches;
                     if (!mbar_wait_warp(smem_u32(&ctl.b_free[bb]), (use & 1) ^ 1, abort_flag, status, 600 + bb)) { ok = false; return; }
@@ -481,6 +527,51 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         bulk_load_1d(bres_base + bb * c.bres_stride + blk * blk_bytes, wtile + (size_t)blk * blk_bytes, blk_bytes, bar);
                     cur_gn = (int)gn;
                     ++switches;
+                }
+                const uint32_t piece_bytes = (uint32_t)c.CK * (uint32_t)c.boxpx * 4u;
+                const uint32_t part_bytes = (uint32_t)c.pieces * piece_bytes;
+                for (int ks = 0; ks < kstages; ++ks, ++it) {
+                    const uint32_t rs = it % (uint32_t)c.raw_stages, ruse = it / (uint32_t)c.raw_stages;
+                    if (ruse > 0 && !mbar_wait_warp(smem_u32(&ctl.raw_empty[rs]), (ruse - 1) & 1u, abort_flag, status, 150 + (int)rs)) { ok = false; break; }
+                    const uint32_t rbar = smem_u32(&ctl.raw_full[rs]);
+                    const uint32_t rdst = smem_base + c.raw_off + rs * c.raw_bytes;
+                    const int chan = g * c.Cg + ks * c.CK;
+                    if (c.raw_bulk) {
+                        // whole planes of CK consecutive channels are one contiguous run of the input tensor
+                        uint32_t live = 0;
+                        for (int pt = 0; pt < c.IPT; ++pt) {
+                            int n, fa;
+                            gath_part(s, c, mt, pt, n, fa);
+                            live += n < s.N ? 1u : 0u;
+                        }
+                        if (lane == 0) mbar_arrive_expect_tx(rbar, live * part_bytes);
+                        __syncwarp();
+                        if (lane < c.IPT) {
+                            int n, fa;
+                            gath_part(s, c, mt, lane, n, fa);
+                            if (n < s.N)
+                                bulk_load_1d(rdst + (uint32_t)lane * part_bytes, x + ((size_t)n * s.C_in + (size_t)chan) * (size_t)HW, part_bytes, rbar);
+                        }
+                    } else {
+                        if (lane == 0) mbar_arrive_expect_tx(rbar, (uint32_t)c.IPT * part_bytes);   // out-of-range boxes arrive as zeros
+                        __syncwarp();
+                        if (lane < c.IPT * c.pieces) {
+                            const int pt = lane / c.pieces, pc = lane - pt * c.pieces;
+                            int n, fa;
+                            gath_part(s, c, mt, pt, n, fa);
+                            tma_load_3d(rdst + (uint32_t)pt * part_bytes + (uint32_t)pc * piece_bytes, &xmap4, fa + pc * c.boxpx, chan, n, rbar);
+                        }
+                    }
+                    if (!c.b_res) {
+                        if (it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                        const uint32_t nb = (uint32_t)c.nr * blk_bytes;
+                        const uint32_t full = smem_u32(&ctl.full[stage]);
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(full, nb);
+                            bulk_load_1d(stage_base + (uint32_t)stage * c.stage_bytes + a_all, wtile + (size_t)ks * nb, nb, full);
+                        }
+                    }
+                    if (++stage == c.stages) { stage = 0; ph ^= 1; }
                 }
                 return;
             }
@@ -606,7 +697,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             // drain: wait (bounded) for the copies of every stage that may still be in flight, so that no bulk copy
             // lands in this CTA's shared memory after it has exited; a drain that runs out too is recorded in the
             // status detail (1000 + stage, 1100 + weight buffer) beside the code of the wait that gave up first
-            for (int i = 0; i < c.stages && i < (int)it; ++i) {
+            // (gather producer: the copies in flight are the raw buffers'; its stage barriers complete by arrivals)
+            for (int i = 0; c.soft && i < c.raw_stages && i < (int)it; ++i) {
+                const uint32_t j = it - 1 - i;
+                if (!mbar_drain(smem_u32(&ctl.raw_full[j % c.raw_stages]), (j / c.raw_stages) & 1, abort_flag)) status->detail = 1200 + (int)(j % c.raw_stages);
+            }
+            for (int i = 0; !c.soft && i < c.stages && i < (int)it; ++i) {
                 const uint32_t j = it - 1 - i;
                 if ((int)j == c.dbg_skip && blockIdx.x == 0) continue;   // the test hook issued nothing for this fill
                 if (!mbar_drain(smem_u32(&ctl.full[j % c.stages]), (j / c.stages) & 1, abort_flag)) status->detail = 1000 + (int)(j % c.stages);
@@ -654,91 +750,163 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 }
             }
         }
-    } else if (c.soft && warp >= kEpi2First) {
-        // ---------------------------------------------------------------- software producer (copy warps)
-        // Widths TMA cannot address (rows that are not a multiple of 16 bytes: 14, 7, ...): the kernel computes on a
-        // virtual zero-padded plane (s.H x s.W, a power-of-two width that divides 32) and these warps build the
-        // stages themselves -- cp.async of 8 bytes (even widths) or 4 bytes from the real rows into exactly the
-        // shared-memory image TMA would have written (32-pixel blocks, 128-byte row per channel, 32-byte chunks
-        // XOR-swizzled by the channel), zero-size copies for the pad columns, the rows outside the plane and the images
-        // past the batch.  Warp j of the four owns segment j of every four-segment block.  A stage is handed to the
-        // tensor core one stage late: after issuing the next stage's copies the warp waits for its own copies of the
-        // previous one (cp.async groups), makes them visible to the async proxy and arrives on the stage's barrier.
-        // Before it blocks on a stage that is still being read it hands over what it holds (a ring of one stage
-        // would otherwise wait for itself).
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        const int pw = warp - kEpi2First;
-        const bool pairs = (c.Wv & 1) == 0;                 // two pixels per copy
-        const int u = pairs ? (lane & 15) : lane;           // copy unit inside the 32-pixel segment
-        const int kfirst = pairs ? (lane >> 4) : 0, kstep = pairs ? 2 : 1;
-        const int wshift = __ffs(s.W) - 1;
-        const size_t plane = (size_t)c.Hv * (size_t)c.Wv;
-        const uint32_t unit_off = pairs ? ((uint32_t)(u >> 2) << 5) + (uint32_t)(u & 3) * 8u : ((uint32_t)(u >> 3) << 5) + (uint32_t)(u & 7) * 4u;
+    } else if (c.soft && warp >= (c.egroups == 1 ? kEpi2First : kMmaWarp3 + 2)) {
+        // ---------------------------------------------------------------- gather producer (copy warps)
+        // Planes the tiled bulk copies cannot bring as operand rows (row length not a multiple of 16 bytes: 14, 7, ...
+        // wide) and small stride-2 planes.  A tile is four segments; a segment is `rps` whole OUTPUT rows laid side by
+        // side in its 32 lanes (lane = row-in-segment * W_out + column), so a pixel's horizontal neighbours are the
+        // neighbouring lanes and nothing is padded.  Warp 0 lands the raw input rows of the tile in the raw ring; copy
+        // warp j builds segment j of every operand block of the stage from them, shared memory to shared memory, in
+        // exactly the image the tensor core expects (32-pixel blocks, 128-byte row per channel, 32-byte chunks
+        // XOR-swizzled by the channel):
+        //   stride 1: three blocks, one per vertical tap r: A_r[lane] = x[p + (r-1)*dil, q]
+        //   stride 2: six blocks, per vertical tap the even and the odd input column of the output pixel:
+        //             A_rE[lane] = x[2p + r - 1, 2q],  A_rO[lane] = x[2p + r - 1, 2q + 1]
+        // rows and columns outside the plane, lanes past the segment's rows and images past the batch are written as
+        // zeros.  Then fence.proxy.async, one arrival per copy warp on the stage barrier, one on the raw buffer's.
+        const int pw = warp - (c.egroups == 1 ? kEpi2First : kMmaWarp3 + 2);
+        const bool g2 = c.soft == 2;
+        // lanes take two adjacent pixels (8-byte accesses) when pixel pairs never straddle a row: the two half-warps
+        // then take alternate channels
+        const bool pairs = !g2 && (s.W & 1) == 0;
+        const int u = pairs ? (lane & 15) : lane;
+        const int kfirst = pairs ? (lane >> 4) : 0;
+        const int l0 = pairs ? 2 * u : lane;                 // first output lane this thread fills
+        uint32_t rr_, q_;
+        c.div_w.divmod((uint32_t)l0, rr_, q_);
+        const int rr = (int)rr_, q = (int)q_;
         const uint32_t unit_chunk = pairs ? (uint32_t)(u >> 2) : (uint32_t)(u >> 3);
         const uint32_t unit_in = pairs ? (uint32_t)(u & 3) * 8u : (uint32_t)(u & 7) * 4u;
-        (void)unit_off;
+        const uint32_t piece_bytes = (uint32_t)c.CK * (uint32_t)c.boxpx * 4u;
+        const uint32_t part_bytes = (uint32_t)c.pieces * piece_bytes;
+        const int dil = s.dilation;
         uint32_t it = 0;
-        int stage = 0, prev_stage = 0;
+        int stage = 0;
         uint32_t ph = 0;
-        bool ok = true, pending = false;                    // pending: prev_stage's copies are issued but not handed over
-        auto hand_over = [&](bool all) {
-            if (all) asm volatile("cp.async.wait_group 0;" ::: "memory");
-            else asm volatile("cp.async.wait_group 1;" ::: "memory");   // every group but the newest
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.full[prev_stage]));
-        };
+        bool ok = true;
         for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile)) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);
-            uint32_t gq = gn, ntq = 0;
-            if (c.NT > 1) c.div_nt.divmod(gn, gq, ntq);
-            uint32_t n, i;
-            c.div_spi.divmod(mt * 4u + (uint32_t)pw, n, i);
-            const bool img_ok = (int)n < s.N;
-            int ch = 0, r = c.pw ? 1 : 0;
+            // this warp's segment: image, segment of the image, part of the raw buffer it reads
+            int n, i, pt;
+            gath_segment(c, mt, pw, n, i, pt);
+            int npart, fa;
+            gath_part(s, c, mt, pt, npart, fa);
+            const int p = i * c.rps + rr;                    // output row of this lane
+            const bool lane_ok = n < s.N && i < c.SPI && rr < c.rps && p < s.H_out;
             for (int ks = 0; ks < kstages; ++ks, ++it) {
-                if (it >= (uint32_t)c.stages) {
-                    const uint32_t bar = smem_u32(&ctl.empty[stage]);
-                    if (!__all_sync(0xffffffffu, mbar_test_wait(bar, ph ^ 1) ? 1 : 0)) {
-                        if (pending) { hand_over(true); pending = false; }
-                        if (!mbar_wait_warp(bar, ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                const uint32_t rs = it % (uint32_t)c.raw_stages, ruse = it / (uint32_t)c.raw_stages;
+                if (!mbar_wait_warp(smem_u32(&ctl.raw_full[rs]), ruse & 1u, abort_flag, status, 160 + (int)rs)) { ok = false; break; }
+                if (it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
+                // Plain shared-memory pointers; a lane with nothing to read loads from the start of its part and stores zeros
+                // (no divergent branches).  Per element the work is one address add, the load, a select and a store with a
+                // constant offset: the swizzled destination of channel k is base[k & 3] + k * 128 bytes, and the four (two)
+                // bases are computed once per block.  A copy warp is alone with this code on its scheduler, so every
+                // instruction saved shortens the stage's critical path directly.
+                const float* __restrict__ rawp = reinterpret_cast<const float*>(smem + c.raw_off + rs * c.raw_bytes + (uint32_t)pt * part_bytes);
+                float* __restrict__ stg = reinterpret_cast<float*>(smem + (uint32_t)c.b_res * c.bres_stride + (uint32_t)stage * c.stage_bytes);
+                const uint32_t seg_f = seg_bytes >> 2;       // floats per 32-pixel block
+                const uint32_t bpx = (uint32_t)c.boxpx;
+                // (a pointwise layer has the centre tap only: one block, and with stride 2 only the even columns)
+                if (!g2) {
+#pragma unroll
+                    for (int r = 0; r < 3; ++r) {
+                        if (c.pw && r != 1) continue;
+                        const int h = p + (r - 1) * dil;
+                        const bool v = lane_ok && h >= 0 && h < s.H;
+                        uint32_t idx = 0;
+                        if (v) {
+                            uint32_t pc, in;
+                            c.div_boxpx.divmod((uint32_t)(h * s.W + q - fa), pc, in);
+                            idx = pc * (uint32_t)c.CK * bpx + in;
+                        }
+                        float* __restrict__ dp = stg + (uint32_t)((c.pw ? 0 : r) * 4 + pw) * seg_f + (unit_in >> 2);
+                        if (pairs) {
+                            // half-warp hw takes channels k = 2 j + hw: k & 3 is hw or hw + 2
+                            const float* __restrict__ sp = rawp + idx + (uint32_t)kfirst * bpx;
+                            float* __restrict__ d0 = dp + (uint32_t)kfirst * 32u + ((unit_chunk ^ (uint32_t)kfirst) << 3);
+                            float* __restrict__ d1 = dp + (uint32_t)kfirst * 32u + ((unit_chunk ^ (uint32_t)(kfirst + 2)) << 3);
+                            const uint32_t bp2 = 2u * bpx;
+#pragma unroll
+                            for (int j0 = 0; j0 < c.CK / 2; j0 += 8) {
+                                float2 t[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (j0 + j < c.CK / 2) t[j] = *reinterpret_cast<const float2*>(sp + (uint32_t)(j0 + j) * bp2);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (j0 + j < c.CK / 2)
+                                        *reinterpret_cast<float2*>((((j0 + j) & 1) ? d1 : d0) + (j0 + j) * 64) = v ? t[j] : make_float2(0.f, 0.f);
+                            }
+                        } else {
+                            const float* __restrict__ sp = rawp + idx;
+                            float* __restrict__ d[4];
+#pragma unroll
+                            for (int m = 0; m < 4; ++m) d[m] = dp + ((unit_chunk ^ (uint32_t)m) << 3);
+#pragma unroll
+                            for (int k0 = 0; k0 < c.CK; k0 += 8) {
+                                float t[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) t[j] = sp[(uint32_t)(k0 + j) * bpx];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) d[(k0 + j) & 3][(k0 + j) * 32] = v ? t[j] : 0.f;
+                            }
+                        }
+                    }
+                } else {
+                    const bool w_even = (s.W & 1) == 0;      // the (even, odd) column pair of an output pixel is 8-byte aligned
+                    const bool odd_ok = 2 * q + 1 < s.W;
+#pragma unroll
+                    for (int r = 0; r < 3; ++r) {
+                        if (c.pw && r != 1) continue;
+                        const int h = 2 * p + r - 1;
+                        const bool v = lane_ok && h >= 0 && h < s.H;
+                        uint32_t idx = 0;
+                        if (v) {
+                            uint32_t pc, in;
+                            c.div_boxpx.divmod((uint32_t)(h * s.W + 2 * q - fa), pc, in);
+                            idx = pc * (uint32_t)c.CK * bpx + in;
+                        }
+                        const float* __restrict__ sp = rawp + idx;
+                        float* __restrict__ dE = stg + (uint32_t)((c.pw ? 0 : r) * 8 + pw) * seg_f + (unit_in >> 2);
+                        float* __restrict__ d[4];
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) d[m] = dE + ((unit_chunk ^ (uint32_t)m) << 3);
+                        const uint32_t oblk = 4u * seg_f;    // the odd-column block sits four segments behind the even one
+                        const uint32_t oo = (v && odd_ok) ? 1u : 0u;
+#pragma unroll
+                        for (int k0 = 0; k0 < c.CK; k0 += 8) {
+                            float e[8], o[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float* a = sp + (uint32_t)(k0 + j) * bpx;
+                                if (w_even) {
+                                    const float2 t = *reinterpret_cast<const float2*>(a);
+                                    e[j] = t.x;
+                                    o[j] = t.y;
+                                } else {
+                                    e[j] = a[0];
+                                    o[j] = a[oo];
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float* de = d[(k0 + j) & 3] + (k0 + j) * 32;
+                                de[0] = v ? e[j] : 0.f;
+                                if (!c.pw) de[oblk] = oo ? o[j] : 0.f;
+                            }
+                        }
                     }
                 }
-                const uint32_t a_dst = stage_base + (uint32_t)stage * c.stage_bytes;
-                const float* xg = x + ((size_t)(img_ok ? n : 0u) * s.C_in + (size_t)((int)gq * c.Cg + ch * c.CK)) * plane;
-                // this warp's 32-pixel blocks of the stage: block pw, pw + 4, ...  A halo stage (rows of one segment) holds
-                // the tile's rows and the rows above and below, block b = padded row b - wseg of the tile; a tap-block
-                // stage holds three shifted copies of the tile, block 4 * tap + segment; else one block per segment
-                const bool halo = c.nr == 3 && !c.tapb;
-                for (int b = pw, kb = 0; b < c.nseg; b += kSoftWarps, ++kb) {
-                    const int f0 = halo ? ((int)i + 4 * kb - c.wseg) * 32 : (int)i * c.seg_fstep + ((c.tapb ? kb : r) - 1) * rstep;
-                    const int f = f0 + (pairs ? 2 * u : u);   // this lane's first pixel in the padded plane
-                    const int row = f >> wshift, col = f & (s.W - 1);
-                    const bool valid = img_ok && f >= 0 && row < c.Hv && col < c.Wv;
-                    const float* src = valid ? xg + (size_t)row * c.Wv + col : x;
-                    const uint32_t nbytes = valid ? (pairs ? 8u : 4u) : 0u;
-                    const uint32_t dseg = a_dst + (uint32_t)b * seg_bytes + unit_in;
-                    if (pairs) {
-                        for (int k = kfirst; k < c.CK; k += kstep)
-                            asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dseg + (uint32_t)k * 128u + ((unit_chunk ^ ((uint32_t)k & 3u)) << 5)),
-                                         "l"(src + (size_t)k * plane), "r"(nbytes) : "memory");
-                    } else {
-                        for (int k = kfirst; k < c.CK; k += kstep)
-                            asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dseg + (uint32_t)k * 128u + ((unit_chunk ^ ((uint32_t)k & 3u)) << 5)),
-                                         "l"(src + (size_t)k * plane), "r"(nbytes) : "memory");
-                    }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&ctl.full[stage]));
+                    mbar_arrive(smem_u32(&ctl.raw_empty[rs]));
                 }
-                asm volatile("cp.async.commit_group;" ::: "memory");
-                if (pending) hand_over(false);
-                pending = true;
-                prev_stage = stage;
-                if (c.nr == 3 || c.pw) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
         }
-        if (pending && ok) hand_over(true);
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp == 1 || warp == kMmaWarp2 || warp >= kMmaWarp3) {
         // ---------------------------------------------------------------- MMA issuers
         // Two warps issue alternate tiles (each owns one TMEM buffer), so the barrier waits and descriptor
@@ -748,6 +916,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         if (lane == 0 && mslot < (uint32_t)c.issuers) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((uint32_t)(c.Np >> 3) << 17) |
                                    ((128u >> 4) << 24);
+            // stride-2 gather stages: the even-column block meets the centre tap (N = Kt), the odd-column block the left and
+            // right taps (N = 2 Kt); the packed columns are ordered (centre, left, right) for this
+            const uint32_t idesc_e = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(c.Kt >> 3) << 17);
+            const uint32_t idesc_o = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(c.Kt >> 2) << 17);
             const uint32_t b_lbo = (uint32_t)(c.Np >> 3) * 128u;   // next 4-channel core matrix along K
             const uint32_t b_kstep = 2u * b_lbo;                   // 8 channels
             // descriptors differ only in the start-address field of the low word
@@ -823,8 +995,13 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         uint32_t al = alo, bl = blo;
 #pragma unroll 4
                         for (int k8 = 0; k8 < k8n; ++k8, al += 64u, bl += bk16) {
-                            umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc, acc);
-                            if (c.pair) umma_tf32_split(d_tmem + (uint32_t)c.Np, al + a_pair16, a_hi, bl, b_hi, idesc, acc);   // same weights, second tile
+                            if (c.soft == 2 && !c.pw) {
+                                umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc_e, acc);
+                                umma_tf32_split(d_tmem + (uint32_t)c.Kt, al + 4u * (seg_bytes >> 4), a_hi, bl + (uint32_t)c.Kt, b_hi, idesc_o, acc);
+                            } else {
+                                umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc, acc);
+                                if (c.pair) umma_tf32_split(d_tmem + (uint32_t)c.Np, al + a_pair16, a_hi, bl, b_hi, idesc, acc);   // same weights, second tile
+                            }
                             acc = 1;
                         }
                     }
@@ -890,9 +1067,24 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             tile_coords(c, (uint32_t)tile, gn, mt);
             if (c.pair) mt = 2u * mt + egroup;               // pair tiles: group e drains the pair's tile e (accumulator e of the buffer)
             uint32_t n, i;
-            int f;
+            int f = 0;
             bool valid;
-            if (c.rowbox) {
+            bool g_left = false, g_right = false;
+            int g_fo = 0;
+            if (c.soft) {
+                // gather tilings: quarter wq is one segment, lane = row-in-segment * W_out + column
+                int gn_, gi_, gp_;
+                gath_segment(c, mt, wq, gn_, gi_, gp_);
+                n = (uint32_t)gn_;
+                uint32_t rr, q;
+                c.div_w.divmod((uint32_t)lane, rr, q);
+                const int p = gi_ * c.rps + (int)rr;
+                valid = gn_ < s.N && gi_ < c.SPI && (int)rr < c.rps && p < s.H_out;
+                g_fo = p * s.W_out + (int)q;
+                const int dl = c.soft == 2 ? 1 : s.dilation;
+                g_left = (int)q >= dl;
+                g_right = c.soft == 2 ? false : (int)q + dl < s.W_out;
+            } else if (c.rowbox) {
                 // quarter wq is segment h = wq % SR of row p0 + wq / SR; the last segment of a two-segment row is
                 // shifted left to end at column W, and each column is stored by the segment that holds both of its
                 // horizontal neighbours
@@ -920,15 +1112,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 f = (int)i * c.R * s.W + l;
                 valid = (l < c.R * s.W) && (f < HW);
             }
-            uint32_t prow, q;
-            c.div_w.divmod((uint32_t)f, prow, q);
-            const int dil = s.dilation;                  // horizontal taps sit dil columns away (dil > 1: segment tilings only)
-            const bool use_left = (int)q >= dil;
-            const bool use_right = (int)q + dil < s.W;
+            uint32_t prow = 0, q = 0;
+            if (!c.soft) c.div_w.divmod((uint32_t)f, prow, q);
+            const int dil = c.soft == 2 ? 1 : s.dilation;   // horizontal taps sit dil columns away (dil > 1: segment and gather tilings only)
+            const bool use_left = c.soft ? g_left : (int)q >= dil;
+            const bool use_right = c.soft ? g_right : (int)q + dil < s.W;
             // s.H x s.W is the (possibly padded) plane the kernel computes on; only the first Hv x Wv pixels exist in y
-            valid = valid && (int)prow < c.Hv && (int)q < c.Wv;
-            int fo = (int)prow * s.W_out + (int)q;       // position in the output plane
-            if (s.stride == 2) {                         // stride 2 keeps the even rows and columns of the stride-1 result
+            if (!c.soft) valid = valid && (int)prow < c.Hv && (int)q < c.Wv;
+            int fo = c.soft ? g_fo : (int)prow * s.W_out + (int)q;       // position in the output plane
+            if (s.stride == 2 && !c.soft) {              // stride 2 keeps the even rows and columns of the stride-1 result
                 valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
                 fo = (int)(prow >> 1) * s.W_out + (int)(q >> 1);
             }
@@ -999,6 +1191,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 float d0[8], d1[8], d2[8];
                 if (c.pw) {                                // one accumulator per filter, nothing to combine
                     tmem_ld8(t0 + (uint32_t)k0, d1);
+                } else if (c.soft == 2) {                  // columns (centre, left, right): the right tap already sits in its own lane (c.pw is handled above)
+                    tmem_ld8(t0 + (uint32_t)k0, d1);
+                    tmem_ld8(t0 + (uint32_t)(Kt + k0), d0);
+                    tmem_ld8(t0 + (uint32_t)(2 * Kt + k0), d2);
                 } else {
                     tmem_ld8(t0 + (uint32_t)k0, d0);
                     tmem_ld8(t0 + (uint32_t)(Kt + k0), d1);
@@ -1008,7 +1204,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     float v = d1[j];
-                    if (!c.pw) {
+                    if (c.soft == 2 && !c.pw) {
+                        const float up = __shfl_up_sync(0xffffffffu, d0[j], 1u);
+                        v += d2[j];
+                        if (add_up) v += up;
+                    } else if (!c.pw) {
                         const float up = __shfl_up_sync(0xffffffffu, d0[j], (unsigned)dil);
                         const float dn = __shfl_down_sync(0xffffffffu, d2[j], (unsigned)dil);
                         if (add_up) v += up;
@@ -1070,9 +1270,9 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     }
 }
 
-// (the copy-warp families run two 480-thread CTAs per SM: at most 68 registers per thread)
+// (the gather families run two 480-thread CTAs per SM: at most 68 registers per thread)
 template <int F>
-__global__ void __launch_bounds__(family(F).soft == 1 ? 32 * (kEpi2First + kSoftWarps) : kThreads, family(F).soft == 1 ? 2 : 1)
+__global__ void __launch_bounds__(family(F).soft >= 1 ? 32 * (kEpi2First + kSoftWarps) : kThreads, family(F).soft >= 1 ? 2 : 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xmap4, const Shape s_in,
                   const IgemmCfg c_in, const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag,
                   const float* __restrict__ x) {
@@ -1123,8 +1323,9 @@ __global__ void igemm_pack_kernel(Shape s, IgemmCfg c, const float* __restrict__
         const int ce = ch * c.CK + k8 * 8 + k2 * 4 + e;   // channel within the merged group
         uint32_t bits = 0;
         if (ncol < ht * c.Kt) {
-            const int ss = ncol / c.Kt;
-            const int ke = nt * c.Kt + (ncol - ss * c.Kt);  // filter within the merged group
+            const int cb = ncol / c.Kt;
+            const int ss = c.soft == 2 ? (cb == 0 ? 1 : (cb == 1 ? 0 : 2)) : cb;   // stride-2 gather: columns ordered (centre, left, right)
+            const int ke = nt * c.Kt + (ncol - cb * c.Kt);  // filter within the merged group
             const int gi = ke / s.Kg;                        // which original group of the merge
             if (ce / s.Cg == gi) {
                 const int ko = (g * c.merge + gi) * s.Kg + (ke - gi * s.Kg);
@@ -1274,15 +1475,135 @@ bool igemm_supported(const Shape& s_any) {
     const IgemmCfg c = igemm_config(s, 148);
     // Dilation: vertical taps are whole-row shifts for any tiling, but the horizontal neighbours dil columns away must
     // lie in the same 32-pixel segment: segment tilings only (rows that divide 32 pixels).
-    if (s.dilation > 1 && !(c.seg_mode && !c.rowbox && c.nr == 1 && !c.tapb)) return false;
+    if (s.dilation > 1 && !(c.soft == 1 || (c.seg_mode && !c.rowbox && c.nr == 1 && !c.tapb))) return false;
     return c.smem_bytes <= (size_t)kMaxDynSmem;   // the smallest pipeline (two stages) must fit
 }
 
 size_t igemm_scratch_bytes(const Shape& s_any) {
     const Shape s = as_3x3(s_any);
     const IgemmGeom ge = igemm_geom(s);
-    if (!ge.padded || igemm_config(s, kLayoutSMs).soft) return 0;   // copy warps read the real rows: no padded copy
+    if (!ge.padded || igemm_config(s_any, kLayoutSMs).soft) return 0;   // the gather producer reads the real rows: no padded copy
     return sizeof(float) * (size_t)s.N * s.C_in * ge.Hp * ge.Wp;
+}
+
+
+// Gather producer (see the copy warps in the kernel): planes whose rows the tiled bulk copies cannot deliver as operand
+// rows (width not a multiple of 4, up to 32) with stride 1, and stride-2 layers on such planes.  Narrow (merged) groups in
+// the two-CTA launch shape.  Fills every field of the configuration; returns false when the shape is not taken.
+static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
+    IgemmCfg c = out;                    // committed only when the shape is taken
+    const int mode = st.stride == 2 ? 2 : 1;
+    if (st.KH != 3 || st.W % 4 == 0 || st.W_out > 32 || st.W_out < 1) return false;
+    if (c.Cg > 32) return false;                                         // narrow (merged) groups only
+    const int vt = c.pw ? 1 : 3;                                         // vertical taps (a pointwise layer has the centre one only)
+    if (!c.pw && 2 * c.Np > 256 && c.Kg % 32 == 0) {                     // two accumulators must fit 256 columns: 32-filter tiles
+        c.Kt = 32;
+        c.NT = c.Kg / 32;
+        c.Np = 96;
+    }
+    if (2 * c.Np > 256) return false;
+    if (mode == 2 && (st.dilation != 1 || c.Kt % 16 != 0)) return false;
+    const uint32_t b_tile = (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u;
+    if (b_tile > 40u * 1024u) return false;
+    c.soft = mode;
+    c.padded = 0;
+    c.Hv = st.H;
+    c.Wv = st.W;
+    c.CK = c.Cg % 16 == 0 ? 16 : 8;
+    c.chunks = c.Cg / c.CK;
+    const int Wo = st.W_out, Ho = st.H_out, HW = st.H * st.W;
+    c.rps = 32 / Wo;
+    c.SPI = (Ho + c.rps - 1) / c.rps;
+    int tpi = 1;
+    if (c.SPI >= 3) {
+        c.IPT = 1;
+        tpi = (c.SPI + 3) / 4;
+        c.MT = st.N * tpi;
+    } else {
+        c.IPT = 4 / c.SPI;
+        c.MT = (st.N + c.IPT - 1) / c.IPT;
+    }
+    c.MTr = c.MT;
+    // raw parts: the input rows a tile needs, as flat pixels from a multiple of 4 on
+    c.raw_bulk = HW % 4 != 0 ? 1 : 0;
+    int px;
+    if (c.raw_bulk) {
+        c.raw_whole = 1;
+        c.pieces = 1;
+        c.boxpx = HW;
+        px = HW;
+    } else {
+        const int rows = st.stride * (4 * c.rps - 1) + 2 * st.dilation + 1;
+        px = rows * st.W + 3;
+        c.raw_whole = (c.IPT > 1 || px >= HW) ? 1 : 0;
+        if (c.raw_whole) px = HW;
+        c.pieces = (px + 255) / 256;
+        c.boxpx = (((px + c.pieces - 1) / c.pieces) + 3) & ~3;
+    }
+    if (c.IPT * c.pieces > 32) return false;
+    c.div_boxpx = make_fastdiv((uint32_t)c.boxpx);
+    c.raw_bytes = (uint32_t)c.IPT * (uint32_t)c.pieces * (uint32_t)c.CK * (uint32_t)c.boxpx * 4u;
+    c.raw_bytes = (c.raw_bytes + 127u) & ~127u;
+    c.seg_mode = 0;
+    c.seg_fstep = 32;
+    c.R = c.RB = 0;
+    c.need_xchg = 0;
+    c.rowbox = c.SR = 0;
+    c.s2h = 0;
+    c.lbo_segs = 1;
+    c.nr = vt;
+    c.wseg = c.pw ? 0 : (mode == 1 ? 4 : 8);
+    c.nseg = c.pw ? 4 : (mode == 1 ? 12 : 24);
+    c.tapb = 0;
+    c.fast4 = 0;
+    c.pair = 0;
+    c.nacc = 2;
+    c.issuers = 2;
+    c.egroups = 1;
+    c.threads = 32 * (kEpi2First + kSoftWarps);
+    c.tmem_cols = 256;
+    c.num_tiles = c.groups * c.NT * c.MT;
+    c.div_mt = make_fastdiv((uint32_t)c.MT);
+    c.div_spi = make_fastdiv((uint32_t)tpi);
+    c.div_w = make_fastdiv((uint32_t)Wo);
+    c.div_nt = make_fastdiv((uint32_t)c.NT);
+    c.bres_stride = (b_tile + 1023u) & ~1023u;
+    c.b_res = 1;
+    c.nt_fast = 0;
+    c.stage_bytes = ((uint32_t)c.nseg * (uint32_t)c.CK * 128u + 1023u) & ~1023u;
+    // two CTAs per SM: the bank, as many stages as there are chunks (at most three, at least two when there is room) and two
+    // or three raw buffers inside 110 KB; a single stage and a single raw buffer as the last resort
+    const uint32_t total = 112u * 1024u - 1024u;          // two CTAs per SM: (228 KB - 2 x 2 KB of static and reserved shared memory) / 2, minus the alignment slack
+    if (c.bres_stride + c.stage_bytes + c.raw_bytes > total) return false;
+    c.stages = 1;
+    c.raw_stages = 1;
+    for (;;) {
+        const uint32_t used = c.bres_stride + (uint32_t)c.stages * c.stage_bytes + (uint32_t)c.raw_stages * c.raw_bytes;
+        if (c.raw_stages <= c.stages && c.raw_stages < 3 && used + c.raw_bytes <= total) { ++c.raw_stages; continue; }
+        if (c.stages < 3 && used + c.stage_bytes <= total) { ++c.stages; continue; }
+        break;
+    }
+    c.raw_off = c.bres_stride + (uint32_t)c.stages * c.stage_bytes;
+    c.xchg_off = c.raw_off + (uint32_t)c.raw_stages * c.raw_bytes;
+    c.smem_bytes = (size_t)c.xchg_off + 1024;
+    c.grid = c.num_tiles < 2 * sm_count ? c.num_tiles : 2 * sm_count;
+    c.cps = 0;
+    c.fuse = 0;
+    c.ball = 0;
+    c.C2 = 0;
+    c.n_gn = c.groups * c.NT;
+    c.div_ngn = make_fastdiv((uint32_t)c.n_gn);
+    c.d2_col = c.nacc * c.Np;
+    c.d2_bufs = 1;
+    c.w2_off = c.a2_off = 0;
+    c.w2_goff = 0;
+    if (c.n_gn > 1 && c.grid >= c.n_gn) {
+        c.cps = c.grid / c.n_gn;                     // CTAs per (group, filter tile): no CTA ever switches weights
+        if (c.cps > c.MT) c.cps = c.MT;
+        c.grid = c.cps * c.n_gn;
+    }
+    out = c;
+    return true;
 }
 
 static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
@@ -1320,6 +1641,11 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.Kt = kt;
     c.NT = c.Kg / kt;
     c.Np = (vt * kt + 15) & ~15;
+    c.soft = 0;
+    c.rps = c.IPT = c.boxpx = c.pieces = c.raw_whole = c.raw_bulk = c.raw_stages = 0;
+    c.raw_off = c.raw_bytes = 0;
+    c.div_boxpx = make_fastdiv(1);
+    if (!fuse && gather_config(c, s_true, sm_count)) return c;
     const int HW = s.H * s.W;
     c.seg_mode = (32 % s.W == 0) && (HW % 32 == 0);
     c.seg_fstep = 32;
@@ -1500,16 +1826,6 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
             budget_total = light_total - 1024u - (fits_fused ? ((w2_bytes + 1023u) & ~1023u) + a2_bytes + 1024u : 0u);
         }
     }
-    // Software producer: a width TMA cannot address whose padded plane is a whole number of segments, in the light
-    // shape.  The copy warps read the real rows, so there is no padded copy of x and no extra launch.
-    // Odd widths copy four bytes at a time, which only pays while the layer is small (measured: 7x7 planes, 3 MB of x
-    // 22 % faster, 13 MB 12 % slower than the padded copy); even widths copy eight and always pay.
-    const bool soft_pays = (s_true.W % 2 == 0) || (size_t)s_true.N * s_true.C_in * s_true.H * s_true.W * 4u <= (8u << 20);
-    c.soft = (ge.padded && c.seg_mode && c.egroups == 1 && !fuse && soft_pays) ? 1 : 0;
-    if (c.soft) {
-        c.padded = 0;
-        c.threads += 32 * kSoftWarps;
-    }
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
     c.stage_bytes = ((c.pair ? 2u : 1u) * a_bytes + (c.b_res ? 0u : (uint32_t)c.nr * blk) + 1023u) & ~1023u;
     if (c.pair) budget_total = 216u * 1024u;          // three 68 KB stages
@@ -1667,11 +1983,6 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
         s.H = ge.Hp;
         s.W = ge.Wp;
         x = scratch;
-    } else if (c.soft) {
-        // the kernel walks the virtual padded plane; its copy warps read the real rows of x (the tensor maps go unused)
-        const IgemmGeom ge = igemm_geom(s);
-        s.H = ge.Hp;
-        s.W = ge.Wp;
     }
     EncodeTiledFn encode = get_encode_fn();
     if (encode == nullptr) return cudaErrorNotSupported;
@@ -1681,17 +1992,30 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
     const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)s.C_in};
     const cuuint32_t box[3] = {32, (cuuint32_t)c.CK, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    if (c.soft) {
+        memset(&xmap, 0, sizeof(xmap));      // the gather producer uses no swizzled map (and odd planes cannot have one)
+    } else {
+        const CUresult r = encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
     // 4-D view for whole-tile copies: (pixel, channel, 32-pixel segment, image); the segment axis re-walks the
     // pixel axis in steps of 128 bytes, so one box covers nseg consecutive segments.
     IgemmCfg cfg = c;
     CUtensorMap xmap4 = xmap;
     cfg.fast4 = 0;
     if (c.soft) {
-        // no second map
+        // gather producer: raw boxes of (boxpx flat pixels, CK channels) of one image, unswizzled; planes that are not a
+        // multiple of 16 bytes are fetched by plain bulk copies instead (no map)
+        if (!c.raw_bulk) {
+            const cuuint32_t boxr[3] = {(cuuint32_t)c.boxpx, (cuuint32_t)c.CK, 1};
+            if (encode(&xmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(x), dims, strides, boxr, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+            cfg.fast4 = 1;   // the second map is in use (prefetch its descriptor)
+        }
     } else if (c.rowbox) {
         // (column, channel, row segment, row, image); the segment axis steps (W - 32) columns
         const cuuint64_t dims5[5] = {(cuuint64_t)s.W, (cuuint64_t)s.C_in, (cuuint64_t)c.SR, (cuuint64_t)s.H, (cuuint64_t)s.N};
@@ -1740,7 +2064,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
                                                 igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
                                                 igemm_tf32_kernel<21>, igemm_tf32_kernel<22>, igemm_tf32_kernel<23>,
-                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>};
+                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>, igemm_tf32_kernel<26>, igemm_tf32_kernel<27>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;

@@ -115,9 +115,9 @@ def test_pair_tile_shapes(cfg):
     assert used == gconv.GCONV_VARIANT_IGEMM_TF32
 
 
-# Widths whose rows are not a multiple of 16 bytes, in the configurations where copy warps (cp.async) build the stages
-# instead of TMA: even widths (8-byte copies) and odd ones (4-byte), padded widths 8, 16 and 32, planes that end inside
-# a tile, batches that end inside a tile, many tiles per CTA, several groups per CTA, stride 2 on 7x7 planes.
+# Widths whose rows are not a multiple of 16 bytes, where the gather producer builds the stages (raw rows by bulk copy,
+# copy warps shared memory to shared memory): even widths (8-byte accesses) and odd ones, planes that end inside a tile,
+# batches that end inside a tile, many tiles per CTA, several groups per CTA, stride 2 on 7x7 planes.
 COPY_WARP_SHAPES = [
     (5, 32, 14, 14, 32, 3, 3, 1, 1, 1, 4), (9, 64, 7, 7, 64, 3, 3, 1, 1, 1, 2), (2, 16, 17, 30, 16, 3, 3, 1, 1, 1, 2),
     (3, 24, 10, 6, 24, 3, 3, 1, 1, 1, 3), (4, 32, 15, 15, 32, 3, 3, 1, 1, 1, 1), (2, 8, 9, 31, 16, 3, 3, 1, 1, 1, 1),
@@ -125,6 +125,33 @@ COPY_WARP_SHAPES = [
     (33, 256, 7, 7, 256, 3, 3, 1, 1, 1, 8), (1, 8, 5, 7, 8, 3, 3, 1, 1, 1, 1), (6, 48, 13, 14, 96, 3, 3, 1, 1, 1, 6),
     (3, 512, 56, 30, 512, 3, 3, 1, 1, 1, 64), (5, 32, 28, 31, 32, 3, 3, 1, 1, 1, 2), (2, 16, 8, 29, 16, 3, 3, 1, 1, 1, 1),   # halo stages
 ]
+
+
+# More of the gather producer: stride 2 (even/odd column blocks) on 14x14, 7x7, 15x15, 30-wide and 13x9 planes, tiles
+# made of two and of four whole images, a tile that is the short last one of its image, whole-plane bulk copies (planes
+# that are not a multiple of 16 bytes) and boxes of a row range, two filter tiles per group, dilation, 8- and
+# 16-channel stages, pointwise layers (centre tap only) with both strides, a batch that ends inside a tile.
+GATHER_SHAPES = [
+    (64, 256, 14, 14, 512, 3, 3, 2, 1, 1, 16), (9, 64, 14, 14, 128, 3, 3, 2, 1, 1, 2), (7, 32, 7, 7, 32, 3, 3, 2, 1, 1, 1),
+    (5, 32, 15, 15, 64, 3, 3, 2, 1, 1, 2), (3, 16, 11, 30, 32, 3, 3, 2, 1, 1, 1), (6, 48, 13, 9, 96, 3, 3, 2, 1, 1, 6),
+    (11, 32, 7, 6, 32, 3, 3, 2, 1, 1, 1), (4, 32, 19, 18, 32, 3, 3, 2, 1, 1, 1), (3, 24, 22, 22, 24, 3, 3, 1, 1, 1, 1),
+    (2, 32, 30, 30, 32, 3, 3, 1, 1, 1, 2), (13, 8, 6, 6, 16, 3, 3, 1, 1, 1, 1), (3, 32, 14, 14, 128, 3, 3, 1, 1, 1, 1),
+    (4, 32, 14, 14, 32, 3, 3, 1, 3, 3, 2), (3, 16, 15, 30, 64, 1, 1, 2, 0, 1, 1), (5, 24, 7, 7, 40, 1, 1, 1, 0, 1, 1),
+    (2, 192, 15, 30, 1024, 1, 1, 2, 0, 1, 8), (33, 256, 14, 14, 512, 3, 3, 2, 1, 1, 8),
+]
+
+
+@pytest.mark.parametrize("cfg", GATHER_SHAPES)
+def test_gather_producer_shapes(cfg):
+    L = Layer("gather", *cfg)
+    d = gconv.gconv_desc_create(*L.desc_args())
+    try:
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32
+        assert gconv.gconv_forward_launches(d) == 1 and gconv.gconv_workspace_bytes(d) == 0
+    finally:
+        gconv.gconv_desc_destroy(d)
+    check_layer(L, seed=27)
+    check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=27)
 
 
 @pytest.mark.parametrize("cfg", COPY_WARP_SHAPES)
