@@ -365,51 +365,54 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     volatile int* abort_flag = &ctl.abort_flag;
     float (*xchg)[4][2][64] = reinterpret_cast<float (*)[4][2][64]>(smem + c.xchg_off);   // edge-lane exchange (flat row tiles only)
 
-    // barrier set-up, one barrier per thread of the last warps (warp 1 is busy allocating TMEM meanwhile)
-    {
-        const int t = (int)threadIdx.x - 64;
-        if (t >= 0 && t < 8) {
-            if (t < c.stages) {
-                mbar_init(smem_u32(&ctl.full[t]), c.soft ? (uint32_t)kSoftWarps + (c.b_res ? 0u : 1u) : 1u);   // copy warps (+ the streamed weights' arm)
-                mbar_init(smem_u32(&ctl.empty[t]), 1);
-            }
-            if (c.soft && t < 4) {
-                mbar_init(smem_u32(&ctl.raw_full[t]), 1);
-                mbar_init(smem_u32(&ctl.raw_empty[t]), kSoftWarps);
-            }
-        } else if (t >= 8 && t < 8 + kMaxAcc) {
-            const int i = t - 8;
-            mbar_init(smem_u32(&ctl.tmem_full[i]), 1);
-            mbar_init(smem_u32(&ctl.tmem_empty[i]), c.pair ? 2u * kEpiWarps : (uint32_t)kEpiWarps);   // pair tiles: both groups drain the buffer
-            mbar_init(smem_u32(&ctl.xchg_bar[i]), kEpiWarps);
-        } else if (t >= 16 && t < 18) {
-            const int i = t - 16;
-            mbar_init(smem_u32(&ctl.b_full[i]), 1);
-            mbar_init(smem_u32(&ctl.b_free[i]), (uint32_t)c.issuers);
-        } else if (t == 18) {
+    // Set-up.  The producer warp initialises every barrier itself and goes straight on to its copies: it needs neither the
+    // tensor-memory address nor anybody else's work, and on a short layer its first copy is the head of the critical path.
+    // It only ARRIVES on the set-up barrier (named barrier 1); the other warps wait there for the barriers and for warp 1's
+    // tensor-memory allocation.
+    if (warp == 0) {
+        // The barriers are consecutive 8-byte words at the head of the control block; lane j initialises numbers j and
+        // j + 32 with a count picked by selects (no divergent branches: this warp is alone on the critical path here).
+        // Barriers a configuration does not use are initialised too; nobody touches them.
+        constexpr int kBarriers = (int)(offsetof(SharedCtl, tmem_base) / 8);
+        static_assert(offsetof(SharedCtl, full) == 0 && kBarriers <= 64, "barriers first, at most two per lane");
+        const uint32_t n_full = c.soft ? (uint32_t)kSoftWarps + (c.b_res ? 0u : 1u) : 1u;   // copy warps (+ the streamed weights' arm)
+        const uint32_t n_tmem_empty = c.pair ? 2u * kEpiWarps : (uint32_t)kEpiWarps;         // pair tiles: both groups drain the buffer
+#pragma unroll
+        for (int round = 0; round < 2; ++round) {
+            const int t = lane + 32 * round;
+            const int w8 = t * 8;                       // byte offset of barrier t
+            uint32_t n = 1u;
+            n = (w8 >= (int)offsetof(SharedCtl, full) && w8 < (int)offsetof(SharedCtl, empty)) ? n_full : n;
+            n = (w8 >= (int)offsetof(SharedCtl, tmem_empty) && w8 < (int)offsetof(SharedCtl, xchg_bar)) ? n_tmem_empty : n;
+            n = (w8 >= (int)offsetof(SharedCtl, xchg_bar) && w8 < (int)offsetof(SharedCtl, b_full)) ? (uint32_t)kEpiWarps : n;
+            n = (w8 >= (int)offsetof(SharedCtl, b_free) && w8 < (int)offsetof(SharedCtl, a2_full)) ? (uint32_t)c.issuers : n;
+            n = (w8 >= (int)offsetof(SharedCtl, a2_full) && w8 < (int)offsetof(SharedCtl, a2_free)) ? (uint32_t)kEpiWarps : n;
+            n = (w8 >= (int)offsetof(SharedCtl, d2_free) && w8 < (int)offsetof(SharedCtl, w2_full)) ? (uint32_t)kEpiWarps : n;
+            n = (w8 >= (int)offsetof(SharedCtl, raw_empty) && w8 < (int)offsetof(SharedCtl, tmem_base)) ? (uint32_t)kSoftWarps : n;
+            if (t < kBarriers) mbar_init(smem_u32(&ctl) + (uint32_t)w8, n);
+        }
+        if (lane == 0) {
             ctl.abort_flag = 0;
             ctl.wait_us = c.wait_us;
-        } else if (c.fuse && t >= 20 && t < 22) {
-            mbar_init(smem_u32(&ctl.a2_full[t - 20]), kEpiWarps);
-            mbar_init(smem_u32(&ctl.a2_free[t - 20]), 1);
-        } else if (c.fuse && t == 22) {
-            mbar_init(smem_u32(&ctl.w2_full), 1);
-        } else if (c.fuse && t >= 24 && t < 26) {
-            mbar_init(smem_u32(&ctl.d2_full[t - 24]), 1);
-            mbar_init(smem_u32(&ctl.d2_free[t - 24]), kEpiWarps);
         }
-        if (t >= 0 && t < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // the bulk copies complete on these barriers through the async proxy and may be issued a few instructions from
+        // here: the initialisations have to be visible to that proxy, not only to the other threads
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        asm volatile("barrier.arrive 1, %0;" ::"r"((uint32_t)blockDim.x) : "memory");
+    } else {
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
+                         "r"((uint32_t)c.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        tc_fence_before();
+        asm volatile("barrier.sync 1, %0;" ::"r"((uint32_t)blockDim.x) : "memory");
+        tc_fence_after();
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
-                     "r"((uint32_t)c.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = ctl.tmem_base;
+    const uint32_t tmem_base = warp == 0 ? 0u : ctl.tmem_base;   // (the producer never touches tensor memory)
     const bool tag_ok = (tag_seen == tag);   // uniform across the CTA
     // Tiles of this CTA: every gridDim.x-th tile, or -- with resident weights and several (group, filter tile) pairs --
     // the CTAs split into one set per pair, each set striding over that pair's pixel tiles: no CTA ever switches
@@ -447,13 +450,17 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     const int rstep = s.W * s.dilation;          // flat-pixel distance between vertical taps
     const size_t OHW = (size_t)s.H_out * s.W_out;
 
+    bool run_epilogue = false;
     if (!tag_ok) {
         // wrong weights: no role runs, y stays untouched; fall through to the common exit (TMEM is freed there)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
-    } else if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
+    } else if (warp == 0 || (warp == 2 && !c.soft)) {
+        // ---------------------------------------------------------------- TMA producer (warp 0)
         // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
+        // Warp 2, an epilogue warp with nothing to do yet, runs the same tile walk once as a prefetch pass (see below) and
+        // then goes on to its epilogue role.
+        const bool producer = warp == 0;
         uint32_t it = 0, switches = 0;
         int stage = 0;
         uint32_t ph = 0;                                   // phase parity of the current pass over the stage ring
@@ -463,7 +470,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
             if (c.fast4 || c.rowbox) asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap4) : "memory");
         }
-        if (c.b_res && tile_first < tile_end) {
+        if (producer && c.b_res && tile_first < tile_end) {
             // The first tile's resident weights do not depend on the previous kernel: fetch them before waiting for it.
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile_first, gn, mt);
@@ -485,7 +492,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 switches = 2;
             }
         }
-        if (c.fuse) {
+        if (producer && c.fuse) {
             // the pointwise weights of every group stay resident (they come from the packing kernel too)
             const uint32_t bar = smem_u32(&ctl.w2_full);
             const uint32_t w2_blk = (uint32_t)c.Kt * (uint32_t)c.C2 * 4u;
@@ -495,12 +502,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 bulk_load_1d(smem_base + c.w2_off + (uint32_t)blk * w2_blk,
                              reinterpret_cast<const uint8_t*>(packed) + c.w2_goff + (size_t)blk * w2_blk, w2_blk, bar);
         }
-        // Two passes over the tiles.  Pass 0 runs before the dependency wait and only asks L2 to fetch the input box of
-        // the first stage: a cache hint, nothing is consumed, and L2 is the point of coherence, so it stays correct if
-        // the previous kernel is still writing those lines (then they are in L2 already).  The CTA usually sits in the
-        // wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2 instead
-        // of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
-        // Pass 1 is the real one.
+        // Two walks over the tiles.  The prefetch walk (warp 2, before its own dependency wait) only asks L2 to fetch the
+        // input box of the first stage: a cache hint, nothing is consumed, and L2 is the point of coherence, so it stays
+        // correct if the previous kernel is still writing those lines (then they are in L2 already).  The CTA usually
+        // sits in the wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2
+        // instead of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
+        // It used to run on the producer warp ahead of the real walk and cost it 1 500 cycles (a single warp walking
+        // branchy code retires an instruction every five to ten cycles) before the first real copy.  The real walk is
+        // the producer's.
         // One tile's stages: the real copies (arming the stage barriers), or -- pf -- only L2 prefetches of the first
         // pf_limit of them (no barrier).  (Asking L2 for the CTA's next tile while the current one is in flight was
         // measured too: 2 % slower on the stack.)
@@ -681,19 +690,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
             }
         };
-        for (int pass = (c.soft ? 1 : 0); pass < 2 && ok; ++pass) {
-        const bool pf = pass == 0;
-        if (!pf) {
+        if (!producer) {
+            for (int tile = tile_first; tile < tile_end && it < kPrefetchUses; tile = tile_next(tile)) visit(tile, true, kPrefetchUses, it, stage, ph);
+            run_epilogue = true;
+        } else {
             asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
-            it = 0;
-            stage = 0;
-            ph = 0;
+            for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile)) visit(tile, false, 0u, it, stage, ph);
         }
-        for (int tile = tile_first; tile < tile_end && ok && !(pf && it >= kPrefetchUses); tile = tile_next(tile)) {
-            visit(tile, pf, kPrefetchUses, it, stage, ph);
-        }
-        }
-        if (!ok && lane == 0) {
+        if (producer && !ok && lane == 0) {
             // drain: wait (bounded) for the copies of every stage that may still be in flight, so that no bulk copy
             // lands in this CTA's shared memory after it has exited; a drain that runs out too is recorded in the
             // status detail (1000 + stage, 1100 + weight buffer) beside the code of the wait that gave up first
@@ -1012,6 +1016,9 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             }
         }
     } else {
+        run_epilogue = true;
+    }
+    if (run_epilogue) {
         // ---------------------------------------------------------------- epilogue warps
         // Two groups of eight warps take alternate tiles, so one tile's TMEM reads, shuffles and stores overlap
         // the next tile's.  With an even number of accumulators a buffer always belongs to the same group.
