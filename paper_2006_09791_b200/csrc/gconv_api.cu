@@ -109,6 +109,7 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
     d->device = -1;
     d->sm_count = 0;
     d->last_cuda_error = 0;
+    d->last_detail = 0;
     d->workspace = nullptr;
     d->workspace_bytes = 0;
     d->pack_epoch_seen = 0;
@@ -299,6 +300,7 @@ int gconv_last_status(gconv_desc_t d, void* stream) {
     e = cudaMemcpy(&h, d->status_dev, sizeof(Status), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail_cuda(d, e);
     if (h.code != 0) {
+        d->last_detail = h.detail;
         e = cudaMemset(d->status_dev, 0, sizeof(Status));
         if (e != cudaSuccess) return fail_cuda(d, e);
     }
@@ -306,6 +308,8 @@ int gconv_last_status(gconv_desc_t d, void* stream) {
 }
 
 int gconv_last_cuda_error(gconv_desc_t d) { return d == nullptr ? 0 : d->last_cuda_error; }
+
+int gconv_last_status_detail(gconv_desc_t d) { return d == nullptr ? 0 : d->last_detail; }
 
 const char* gconv_status_string(int status) {
     switch (status) {

@@ -23,6 +23,7 @@ struct gconv_desc {
     int device;                  // device the status block lives on (-1 = none yet)
     int sm_count;
     int last_cuda_error;
+    int last_detail;             // detail word that came with the last non-zero device status (which wait, which thread block)
     float* workspace;            // caller-owned device workspace attached by gconv_desc_set_workspace (nullptr = none)
     size_t workspace_bytes;
     unsigned long long pack_epoch_seen;   // value of the process-wide pack counter at this descriptor's last forward

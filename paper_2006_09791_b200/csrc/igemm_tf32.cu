@@ -56,7 +56,8 @@ constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 // Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
 constexpr int kLayoutSMs = 148;
-constexpr uint32_t kPrefetchUses = 1;   // stages whose input is prefetched into L2 before the dependency wait
+constexpr uint32_t kPrefetchUses = 2;   // stage fills (from the CTA's first on) whose input idle epilogue warps ask L2 for before the dependency wait
+                                        // (measured on the 90-launch stack: none 0.660 ms, one 0.610, two 0.597, three 0.602, four 0.611, eight 0.619)
 constexpr uint32_t kDefaultWaitUs = 1000000u;   // a wait gives up after one second unless the descriptor says otherwise
 constexpr int kMaxDynSmem = 226 * 1024;   // 227 KB per CTA minus the static control block (under 1 KB)
 
@@ -122,15 +123,26 @@ __device__ __forceinline__ uint64_t global_ns() {
 
 // Bounded wait: gives up after the CTA's time limit (one second by default).  Returns false if the wait ran out or
 // another role already gave up; the first role to run out records GCONV_ERR_TIMEOUT with `where` as the detail.
+//
+// The polls follow each other as closely as they can.  Some waiters only OBSERVE a barrier that others drive (an MMA warp
+// walking the other warp's stages, see there): a parity wait is only meaningful one phase at a time, so such a waiter must
+// never be away from the barrier for as long as two phase flips take (a refill is a microsecond or more away).  The clock
+// (a read of the global timer is slow) is therefore looked at only once every 128 polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, Status* status,
                                           int where) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t limit_ns = 1000ull * (uint64_t)(uint32_t)abort_flag[1];
-    const uint64_t t0 = global_ns();
+    uint64_t limit_ns = 0, t0 = 0;
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_ns() - t0 > limit_ns) break;
+        if ((it & 127u) == 127u) {
+            if (it == 127u) {
+                limit_ns = 1000ull * (uint64_t)(uint32_t)abort_flag[1];
+                t0 = global_ns();
+            } else if (global_ns() - t0 > limit_ns) {
+                break;
+            }
+        }
         if (it > 4096) __nanosleep(64);
     }
     *abort_flag = 1;
@@ -383,6 +395,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             const int w8 = t * 8;                       // byte offset of barrier t
             uint32_t n = 1u;
             n = (w8 >= (int)offsetof(SharedCtl, full) && w8 < (int)offsetof(SharedCtl, empty)) ? n_full : n;
+            n = (w8 >= (int)offsetof(SharedCtl, empty) && w8 < (int)offsetof(SharedCtl, tmem_full)) ? (uint32_t)c.issuers : n;   // the consumer's MMAs and every observer
             n = (w8 >= (int)offsetof(SharedCtl, tmem_empty) && w8 < (int)offsetof(SharedCtl, xchg_bar)) ? n_tmem_empty : n;
             n = (w8 >= (int)offsetof(SharedCtl, xchg_bar) && w8 < (int)offsetof(SharedCtl, b_full)) ? (uint32_t)kEpiWarps : n;
             n = (w8 >= (int)offsetof(SharedCtl, b_free) && w8 < (int)offsetof(SharedCtl, a2_full)) ? (uint32_t)c.issuers : n;
@@ -455,7 +468,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // wrong weights: no role runs, y stays untouched; fall through to the common exit (TMEM is freed there)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (threadIdx.x == 0) record_status(status, GCONV_ERR_PACK_MISMATCH, (int)blockIdx.x);
-    } else if (warp == 0 || (warp == 2 && !c.soft)) {
+    } else if (warp == 0 || (warp >= 2 && warp < 2 + kEpiWarps && !c.soft)) {
         // ---------------------------------------------------------------- TMA producer (warp 0)
         // The whole warp walks the tiles; lane j issues the copy of segment j, lane 0 arms the barriers.
         // Warp 2, an epilogue warp with nothing to do yet, runs the same tile walk once as a prefetch pass (see below) and
@@ -506,10 +519,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // input box of the first stage: a cache hint, nothing is consumed, and L2 is the point of coherence, so it stays
         // correct if the previous kernel is still writing those lines (then they are in L2 already).  The CTA usually
         // sits in the wait while the previous kernel's last CTAs finish; the first copy after the wait then comes from L2
-        // instead of starting a DRAM round trip.  More than one stage costs more issue time than it hides (measured).
-        // It used to run on the producer warp ahead of the real walk and cost it 1 500 cycles (a single warp walking
-        // branchy code retires an instruction every five to ten cycles) before the first real copy.  The real walk is
-        // the producer's.
+        // instead of starting a DRAM round trip.  The walk used to run on the producer warp ahead of the real one and cost
+        // it 1 500 cycles (a single warp walking branchy code retires an instruction every five to ten cycles) before the
+        // first real copy; now the epilogue warps of the first group share it (warp 2 + j takes fill j).  Asking for more
+        // than two fills competes with the previous kernel's own traffic and loses again (kPrefetchUses).  The real walk
+        // is the producer's.
         // One tile's stages: the real copies (arming the stage barriers), or -- pf -- only L2 prefetches of the first
         // pf_limit of them (no barrier).  (Asking L2 for the CTA's next tile while the current one is in flight was
         // measured too: 2 % slower on the stack.)
@@ -614,6 +628,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             int ch = 0, r = (c.nr == 3 || c.pw) ? 1 : 0;   // r = 1: the centre tap (row offset 0)
             for (int ks = 0; ks < kstages; ++ks, ++it) {
                 if (pf && it >= pf_limit) break;
+                if (pf && (it & (uint32_t)(kEpiWarps - 1)) != (uint32_t)(warp - 2)) {   // the prefetch walk is shared: warp 2 + j takes fills j, j + 8, ...
+                    if (c.nr == 3 || c.pw) { ++ch; } else if (++r == 3) { r = 0; ++ch; }
+                    continue;
+                }
                 // the first pass over the ring finds every stage free
                 if (!pf && it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 const uint32_t full = smem_u32(&ctl.full[stage]);
@@ -975,10 +993,14 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     ++switches;
                 }
                 if (!mine) {
-                    // The other warp's tile: observe its stages' phases in order (no MMAs, no release) so that
-                    // this warp's own parity waits never alias a phase it has not seen.
+                    // The other warp's tile: observe its stages' phases in order (no MMAs) so that this warp's own parity
+                    // waits never alias a phase it has not seen -- and tell the producer so: a stage is refilled only when
+                    // its consumer's MMAs have completed AND every other issuing warp has seen the fill.  Without that
+                    // arrival a warp held up on one stage (its copy arriving late, say from DRAM while the others hit L2)
+                    // could miss two flips of another stage and wait for ever on a phase that has long passed.
                     for (int ks = 0; ks < kstages && ok; ++ks) {
                         if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 800 + stage)) ok = false;
+                        else mbar_arrive(smem_u32(&ctl.empty[stage]));
                         if (++stage == c.stages) { stage = 0; ph ^= 1; }
                     }
                     continue;

@@ -57,6 +57,7 @@ _SIGNATURES = {
     "gconv_desc_set_debug": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
     "gconv_last_status": (ctypes.c_int, [_vp, _vp]),
     "gconv_last_cuda_error": (ctypes.c_int, [_vp]),
+    "gconv_last_status_detail": (ctypes.c_int, [_vp]),
     "gconv_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "gconv_variant_name": (ctypes.c_char_p, [ctypes.c_int]),
 }
@@ -217,3 +218,7 @@ def gconv_last_status(desc, stream=None) -> int:
 
 def gconv_last_cuda_error(desc) -> int:
     return int(load().gconv_last_cuda_error(desc))
+
+
+def gconv_last_status_detail(desc) -> int:
+    return int(load().gconv_last_status_detail(desc))

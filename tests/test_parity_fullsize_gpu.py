@@ -124,7 +124,8 @@ def test_more_than_2_to_31_elements():
             y = torch.full((L.y_elems,), float("nan"), dtype=torch.float32, device=dev)
             gconv.gconv_pack_weights(d, torch.from_numpy(w).to(dev), wp)
             gconv.gconv_forward(d, x, wp, y)
-            assert gconv.gconv_last_status(d) == gconv.GCONV_OK
+            st = gconv.gconv_last_status(d)
+            assert st == gconv.GCONV_OK, (gconv.status_string(st), gconv.gconv_last_status_detail(d))
             v = gconv.gconv_variant(d)
             tol = gconv.VARIANT_TOLERANCE[v]
             yv = y.view(N, L.C_out, L.H_out, L.W_out)
