@@ -51,7 +51,8 @@ constexpr int kMmaWarp2 = 2 + kEpiWarps;     // second MMA-issuing warp (the fir
 constexpr int kEpi2First = kMmaWarp2 + 1;    // first warp of the second epilogue group
 constexpr int kMmaWarp3 = kEpi2First + kEpiWarps;   // third and fourth MMA-issuing warps (used when four accumulators fit)
 constexpr int kThreads = 32 * (kMmaWarp3 + 2);
-constexpr int kSoftWarps = 4;        // copy warps of the gather producer, one per segment of a tile: warps kEpi2First ... in the light shape
+constexpr int kSoftWarps = 4;        // copy warps of the gather producer, one per segment of a tile: warps kEpi2First ... in the light shape;
+                                     // the heavy shape has twice as many (two per segment, half of a stage's channels each)
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;               // accumulator buffers in TMEM (ring), as many as fit 512 columns
 // Decisions that shape the packed weights use this SM count, not the device's, so that packing and forward agree.
@@ -306,7 +307,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 28;
+constexpr int kFamilies = 30;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -336,6 +337,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 25 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 16, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9, -1,  1,  0,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights, 16-channel stages
          : f == 26 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  1,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  4,  12,  0, -1,  0,  0,  0,  1,  0,  0}     // gather producer, stride 1, 8-channel stages
          : f == 27 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  2,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  8,  24,  0, -1,  0,  0,  0,  2,  0,  0}     // gather producer, stride 2, 8-channel stages
+         : f == 28 ? Family{0,   0,  3,  0,  -1,  2,  0,  1,  1, 16, -1, 64, 192, -1,  2,  2,  0, -1,  4,  12,  0, -1,  0,  0,  0,  1,  0,  0}     // gather producer, stride 1, wide groups (one CTA per SM, 29 warps)
+         : f == 29 ? Family{0,   0,  3,  0,  -1,  2,  0,  1,  2, 16, -1, 64, 192, -1,  2,  2,  0, -1,  8,  24,  0, -1,  0,  0,  0,  2,  0,  0}     // gather producer, stride 2, wide groups
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -387,7 +390,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // Barriers a configuration does not use are initialised too; nobody touches them.
         constexpr int kBarriers = (int)(offsetof(SharedCtl, tmem_base) / 8);
         static_assert(offsetof(SharedCtl, full) == 0 && kBarriers <= 64, "barriers first, at most two per lane");
-        const uint32_t n_full = c.soft ? (uint32_t)kSoftWarps + (c.b_res ? 0u : 1u) : 1u;   // copy warps (+ the streamed weights' arm)
+        const uint32_t n_copy = (uint32_t)kSoftWarps * (uint32_t)c.egroups;                 // copy warps of the gather producer
+        const uint32_t n_full = c.soft ? n_copy + (c.b_res ? 0u : 1u) : 1u;                 // copy warps (+ the streamed weights' arm)
         const uint32_t n_tmem_empty = c.pair ? 2u * kEpiWarps : (uint32_t)kEpiWarps;         // pair tiles: both groups drain the buffer
 #pragma unroll
         for (int round = 0; round < 2; ++round) {
@@ -401,7 +405,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             n = (w8 >= (int)offsetof(SharedCtl, b_free) && w8 < (int)offsetof(SharedCtl, a2_full)) ? (uint32_t)c.issuers : n;
             n = (w8 >= (int)offsetof(SharedCtl, a2_full) && w8 < (int)offsetof(SharedCtl, a2_free)) ? (uint32_t)kEpiWarps : n;
             n = (w8 >= (int)offsetof(SharedCtl, d2_free) && w8 < (int)offsetof(SharedCtl, w2_full)) ? (uint32_t)kEpiWarps : n;
-            n = (w8 >= (int)offsetof(SharedCtl, raw_empty) && w8 < (int)offsetof(SharedCtl, tmem_base)) ? (uint32_t)kSoftWarps : n;
+            n = (w8 >= (int)offsetof(SharedCtl, raw_empty) && w8 < (int)offsetof(SharedCtl, tmem_base)) ? n_copy : n;
             if (t < kBarriers) mbar_init(smem_u32(&ctl) + (uint32_t)w8, n);
         }
         if (lane == 0) {
@@ -786,7 +790,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         //             A_rE[lane] = x[2p + r - 1, 2q],  A_rO[lane] = x[2p + r - 1, 2q + 1]
         // rows and columns outside the plane, lanes past the segment's rows and images past the batch are written as
         // zeros.  Then fence.proxy.async, one arrival per copy warp on the stage barrier, one on the raw buffer's.
-        const int pw = warp - (c.egroups == 1 ? kEpi2First : kMmaWarp3 + 2);
+        // copy warp j builds segment j & 3; in the heavy shape warps 4..7 take the second half of the stage's channels
+        const int gw = warp - (c.egroups == 1 ? kEpi2First : kMmaWarp3 + 2);
+        const int pw = gw & 3;
+        const int kcount = c.egroups == 2 ? c.CK / 2 : c.CK;            // channels of the stage this warp copies
+        const uint32_t kbase = (uint32_t)(gw >> 2) * (uint32_t)kcount;  // (a multiple of 4: the swizzle term k & 3 is unchanged)
         const bool g2 = c.soft == 2;
         // lanes take two adjacent pixels (8-byte accesses) when pixel pairs never straddle a row: the two half-warps
         // then take alternate channels
@@ -845,28 +853,28 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         float* __restrict__ dp = stg + (uint32_t)((c.pw ? 0 : r) * 4 + pw) * seg_f + (unit_in >> 2);
                         if (pairs) {
                             // half-warp hw takes channels k = 2 j + hw: k & 3 is hw or hw + 2
-                            const float* __restrict__ sp = rawp + idx + (uint32_t)kfirst * bpx;
-                            float* __restrict__ d0 = dp + (uint32_t)kfirst * 32u + ((unit_chunk ^ (uint32_t)kfirst) << 3);
-                            float* __restrict__ d1 = dp + (uint32_t)kfirst * 32u + ((unit_chunk ^ (uint32_t)(kfirst + 2)) << 3);
+                            const float* __restrict__ sp = rawp + idx + ((uint32_t)kfirst + kbase) * bpx;
+                            float* __restrict__ d0 = dp + ((uint32_t)kfirst + kbase) * 32u + ((unit_chunk ^ (uint32_t)kfirst) << 3);
+                            float* __restrict__ d1 = dp + ((uint32_t)kfirst + kbase) * 32u + ((unit_chunk ^ (uint32_t)(kfirst + 2)) << 3);
                             const uint32_t bp2 = 2u * bpx;
 #pragma unroll
-                            for (int j0 = 0; j0 < c.CK / 2; j0 += 8) {
+                            for (int j0 = 0; j0 < kcount / 2; j0 += 8) {
                                 float2 t[8];
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
-                                    if (j0 + j < c.CK / 2) t[j] = *reinterpret_cast<const float2*>(sp + (uint32_t)(j0 + j) * bp2);
+                                    if (j0 + j < kcount / 2) t[j] = *reinterpret_cast<const float2*>(sp + (uint32_t)(j0 + j) * bp2);
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
-                                    if (j0 + j < c.CK / 2)
+                                    if (j0 + j < kcount / 2)
                                         *reinterpret_cast<float2*>((((j0 + j) & 1) ? d1 : d0) + (j0 + j) * 64) = v ? t[j] : make_float2(0.f, 0.f);
                             }
                         } else {
-                            const float* __restrict__ sp = rawp + idx;
+                            const float* __restrict__ sp = rawp + idx + kbase * bpx;
                             float* __restrict__ d[4];
 #pragma unroll
-                            for (int m = 0; m < 4; ++m) d[m] = dp + ((unit_chunk ^ (uint32_t)m) << 3);
+                            for (int m = 0; m < 4; ++m) d[m] = dp + kbase * 32u + ((unit_chunk ^ (uint32_t)m) << 3);
 #pragma unroll
-                            for (int k0 = 0; k0 < c.CK; k0 += 8) {
+                            for (int k0 = 0; k0 < kcount; k0 += 8) {
                                 float t[8];
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) t[j] = sp[(uint32_t)(k0 + j) * bpx];
@@ -889,15 +897,15 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                             c.div_boxpx.divmod((uint32_t)(h * s.W + 2 * q - fa), pc, in);
                             idx = pc * (uint32_t)c.CK * bpx + in;
                         }
-                        const float* __restrict__ sp = rawp + idx;
+                        const float* __restrict__ sp = rawp + idx + kbase * bpx;
                         float* __restrict__ dE = stg + (uint32_t)((c.pw ? 0 : r) * 8 + pw) * seg_f + (unit_in >> 2);
                         float* __restrict__ d[4];
 #pragma unroll
-                        for (int m = 0; m < 4; ++m) d[m] = dE + ((unit_chunk ^ (uint32_t)m) << 3);
+                        for (int m = 0; m < 4; ++m) d[m] = dE + kbase * 32u + ((unit_chunk ^ (uint32_t)m) << 3);
                         const uint32_t oblk = 4u * seg_f;    // the odd-column block sits four segments behind the even one
                         const uint32_t oo = (v && odd_ok) ? 1u : 0u;
 #pragma unroll
-                        for (int k0 = 0; k0 < c.CK; k0 += 8) {
+                        for (int k0 = 0; k0 < kcount; k0 += 8) {
                             float e[8], o[8];
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
@@ -1299,9 +1307,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
     }
 }
 
-// (the gather families run two 480-thread CTAs per SM: at most 68 registers per thread)
+// (the narrow-group gather families run two 480-thread CTAs per SM: at most 68 registers per thread; the wide-group ones run
+// one CTA of 928 threads: at most 70)
 template <int F>
-__global__ void __launch_bounds__(family(F).soft >= 1 ? 32 * (kEpi2First + kSoftWarps) : kThreads, family(F).soft >= 1 ? 2 : 1)
+__global__ void __launch_bounds__(family(F).soft >= 1 ? (family(F).egroups == 2 ? 32 * (kMmaWarp3 + 2 + 2 * kSoftWarps) : 32 * (kEpi2First + kSoftWarps)) : kThreads,
+                                  family(F).soft >= 1 && family(F).egroups == 1 ? 2 : 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xmap4, const Shape s_in,
                   const IgemmCfg c_in, const uint32_t* __restrict__ packed, float* __restrict__ y, Status* status, uint32_t tag,
                   const float* __restrict__ x) {
@@ -1523,17 +1533,21 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     IgemmCfg c = out;                    // committed only when the shape is taken
     const int mode = st.stride == 2 ? 2 : 1;
     if (st.KH != 3 || st.W % 4 == 0 || st.W_out > 32 || st.W_out < 1) return false;
-    if (c.Cg > 32) return false;                                         // narrow (merged) groups only
     const int vt = c.pw ? 1 : 3;                                         // vertical taps (a pointwise layer has the centre one only)
-    if (!c.pw && 2 * c.Np > 256 && c.Kg % 32 == 0) {                     // two accumulators must fit 256 columns: 32-filter tiles
+    // Two launch shapes, as for the other producers: narrow (merged) groups run two CTAs per SM with a small resident bank;
+    // wide groups (more than 32 channels) run one CTA per SM with 29 warps (eight copy warps behind the two epilogue
+    // groups, two per segment), 16-channel stages and the bank resident (up to 144 KB) or streamed with the stages.
+    const bool heavy = c.Cg > 32;
+    if (heavy && (c.pw || c.Cg % 16 != 0 || c.Kt != 64 || st.dilation != 1)) return false;   // (what its two instantiations fix)
+    if (!heavy && !c.pw && 2 * c.Np > 256 && c.Kg % 32 == 0) {           // two accumulators must fit 256 columns: 32-filter tiles
         c.Kt = 32;
         c.NT = c.Kg / 32;
         c.Np = 96;
     }
-    if (2 * c.Np > 256) return false;
+    if (2 * c.Np > (heavy ? 512 : 256)) return false;
     if (mode == 2 && (st.dilation != 1 || c.Kt % 16 != 0)) return false;
     const uint32_t b_tile = (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u;
-    if (b_tile > 40u * 1024u) return false;
+    if (!heavy && b_tile > 40u * 1024u) return false;
     c.soft = mode;
     c.padded = 0;
     c.Hv = st.H;
@@ -1588,34 +1602,43 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     c.pair = 0;
     c.nacc = 2;
     c.issuers = 2;
-    c.egroups = 1;
-    c.threads = 32 * (kEpi2First + kSoftWarps);
-    c.tmem_cols = 256;
+    c.egroups = heavy ? 2 : 1;
+    c.threads = heavy ? 32 * (kMmaWarp3 + 2 + 2 * kSoftWarps) : 32 * (kEpi2First + kSoftWarps);
+    c.tmem_cols = heavy ? 512 : 256;
     c.num_tiles = c.groups * c.NT * c.MT;
     c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)tpi);
     c.div_w = make_fastdiv((uint32_t)Wo);
     c.div_nt = make_fastdiv((uint32_t)c.NT);
     c.bres_stride = (b_tile + 1023u) & ~1023u;
+    const uint32_t a_stage = ((uint32_t)c.nseg * (uint32_t)c.CK * 128u + 1023u) & ~1023u;
+    // two CTAs per SM: (228 KB - 2 x 2 KB of static and reserved shared memory) / 2, minus the alignment slack; one CTA: 226 KB
+    const uint32_t total = heavy ? (uint32_t)kMaxDynSmem - 1024u : 112u * 1024u - 1024u;
+    // the bank stays resident when it leaves room for two stages and two raw buffers, and (a large bank) when a CTA reuses
+    // it over at least two pixel tiles; otherwise its blocks stream with the stages
     c.b_res = 1;
-    c.nt_fast = 0;
-    c.stage_bytes = ((uint32_t)c.nseg * (uint32_t)c.CK * 128u + 1023u) & ~1023u;
-    // two CTAs per SM: the bank, as many stages as there are chunks (at most three, at least two when there is room) and two
-    // or three raw buffers inside 110 KB; a single stage and a single raw buffer as the last resort
-    const uint32_t total = 112u * 1024u - 1024u;          // two CTAs per SM: (228 KB - 2 x 2 KB of static and reserved shared memory) / 2, minus the alignment slack
-    if (c.bres_stride + c.stage_bytes + c.raw_bytes > total) return false;
+    if (heavy && (b_tile > 144u * 1024u || c.bres_stride + 2u * a_stage + 2u * c.raw_bytes > total || c.MT < 2 * sm_count)) c.b_res = 0;
+    c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
+    c.stage_bytes = (a_stage + (c.b_res ? 0u : (uint32_t)c.nr * (uint32_t)c.Np * (uint32_t)c.CK * 4u) + 1023u) & ~1023u;
+    const uint32_t bank = c.b_res ? c.bres_stride : 0u;
+    // the bank, then stages and raw buffers in turn (at most four and four) while they fit; a single stage and a single raw
+    // buffer as the last resort
+    if (bank + c.stage_bytes + c.raw_bytes > total) return false;
     c.stages = 1;
     c.raw_stages = 1;
+    const int max_ring = heavy ? 4 : 3;
     for (;;) {
-        const uint32_t used = c.bres_stride + (uint32_t)c.stages * c.stage_bytes + (uint32_t)c.raw_stages * c.raw_bytes;
-        if (c.raw_stages <= c.stages && c.raw_stages < 3 && used + c.raw_bytes <= total) { ++c.raw_stages; continue; }
-        if (c.stages < 3 && used + c.stage_bytes <= total) { ++c.stages; continue; }
+        const uint32_t used = bank + (uint32_t)c.stages * c.stage_bytes + (uint32_t)c.raw_stages * c.raw_bytes;
+        if (c.raw_stages <= c.stages && c.raw_stages < max_ring && used + c.raw_bytes <= total) { ++c.raw_stages; continue; }
+        if (c.stages < max_ring && used + c.stage_bytes <= total) { ++c.stages; continue; }
         break;
     }
-    c.raw_off = c.bres_stride + (uint32_t)c.stages * c.stage_bytes;
+    if (heavy && c.stages < 2) return false;
+    c.raw_off = bank + (uint32_t)c.stages * c.stage_bytes;
     c.xchg_off = c.raw_off + (uint32_t)c.raw_stages * c.raw_bytes;
     c.smem_bytes = (size_t)c.xchg_off + 1024;
-    c.grid = c.num_tiles < 2 * sm_count ? c.num_tiles : 2 * sm_count;
+    const int ctas = heavy ? sm_count : 2 * sm_count;
+    c.grid = c.num_tiles < ctas ? c.num_tiles : ctas;
     c.cps = 0;
     c.fuse = 0;
     c.ball = 0;
@@ -1626,7 +1649,7 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     c.d2_bufs = 1;
     c.w2_off = c.a2_off = 0;
     c.w2_goff = 0;
-    if (c.n_gn > 1 && c.grid >= c.n_gn) {
+    if (c.b_res && c.n_gn > 1 && c.grid >= c.n_gn) {
         c.cps = c.grid / c.n_gn;                     // CTAs per (group, filter tile): no CTA ever switches weights
         if (c.cps > c.MT) c.cps = c.MT;
         c.grid = c.cps * c.n_gn;
@@ -2093,11 +2116,12 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
                                                 igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
                                                 igemm_tf32_kernel<21>, igemm_tf32_kernel<22>, igemm_tf32_kernel<23>,
-                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>, igemm_tf32_kernel<26>, igemm_tf32_kernel<27>};
+                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>, igemm_tf32_kernel<26>, igemm_tf32_kernel<27>, igemm_tf32_kernel<28>, igemm_tf32_kernel<29>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;
     if (cfg.pair && family(fam).pair != 1) return cudaErrorInvalidValue;   // the generic instantiation has no pair-tile code
+    if (cfg.soft && cfg.egroups == 2 && family(fam).soft != cfg.soft) return cudaErrorInvalidValue;   // 29 warps: only the wide-group gather instantiations take them
     static bool attr_set[64][kFamilies] = {};
     int dev = 0;
     cudaGetDevice(&dev);

@@ -622,10 +622,10 @@ def test_bounded_wait_runs_out_and_the_context_survives():
 
 
 def test_padded_copy_layers_need_an_attached_workspace():
-    """Widths the bulk tensor copies cannot address with groups the copy warps do not serve: gconv_forward allocates
-    nothing, it refuses to run until the caller attaches the workspace, then runs in two launches."""
+    """Widths the bulk tensor copies cannot address that are too wide for the gather producer (more than 32 output columns):
+    gconv_forward allocates nothing, it refuses to run until the caller attaches the workspace, then runs in two launches."""
     dev = torch.device("cuda:0")
-    L = Layer("w18", 3, 128, 18, 18, 128, groups=1)
+    L = Layer("w54", 3, 128, 10, 54, 128, groups=1)
     d = gconv.gconv_desc_create(*L.desc_args())
     try:
         need = gconv.gconv_workspace_bytes(d)

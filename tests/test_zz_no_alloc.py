@@ -55,7 +55,7 @@ def test_static_scratch_matches_on_two_calls_in_a_row():
     # over the first call's leftovers in the shared scratch; the third needs the padded-copy workspace where the
     # build still uses one; the last repeats the first)
     for L, seed in [(Layer("a", 4, 64, 32, 32, 64, groups=2), 11), (Layer("b", 3, 24, 20, 28, 24, stride=2, groups=24), 12),
-                    (Layer("c", 3, 128, 18, 18, 128), 14), (Layer("a", 4, 64, 32, 32, 64, groups=2), 13)]:
+                    (Layer("c", 3, 128, 10, 54, 128), 14), (Layer("a", 4, 64, 32, 32, 64, groups=2), 13)]:
         y_ref, y_new, y_orc, tol = _both_ways(L, seed)
         assert np.all(np.isfinite(y_new))
         scale = float(np.max(np.abs(y_orc)))
