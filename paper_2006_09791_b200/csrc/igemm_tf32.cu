@@ -307,7 +307,7 @@ struct Family {
     int rowbox, seg_mode, nr, need_xchg, b_res, egroups, s2h, lbo_segs, stride, CK, chunks, Kt, Np, NT, nacc, issuers, padded,
         nt_fast, wseg, nseg, SR, fast4, tapb, fuse, ball, soft, pw, pair;   // (pair: 0 where a row leaves it out)
 };
-constexpr int kFamilies = 30;
+constexpr int kFamilies = 31;
 __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
@@ -338,7 +338,8 @@ __host__ __device__ constexpr Family family(int f) {
          : f == 26 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  1,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  4,  12,  0, -1,  0,  0,  0,  1,  0,  0}     // gather producer, stride 1, 8-channel stages
          : f == 27 ? Family{0,   0,  3,  0,   1,  1,  0,  1,  2,  8, -1, -1,  -1, -1,  2,  2,  0,  0,  8,  24,  0, -1,  0,  0,  0,  2,  0,  0}     // gather producer, stride 2, 8-channel stages
          : f == 28 ? Family{0,   0,  3,  0,  -1,  2,  0,  1,  1, 16, -1, 64, 192, -1,  2,  2,  0, -1,  4,  12,  0, -1,  0,  0,  0,  1,  0,  0}     // gather producer, stride 1, wide groups (one CTA per SM, 29 warps)
-         : f == 29 ? Family{0,   0,  3,  0,  -1,  2,  0,  1,  2, 16, -1, 64, 192, -1,  2,  2,  0, -1,  8,  24,  0, -1,  0,  0,  0,  2,  0,  0}     // gather producer, stride 2, wide groups
+         : f == 29 ? Family{0,   0,  3,  0,   0,  2,  0,  1,  2,  8, -1, 64, 192, -1,  1,  1,  0, -1,  8,  24,  0, -1,  0,  0,  0,  2,  0,  1}     // gather producer, stride 2, wide groups, 8-channel stages, streamed weights shared by a pair of pixel tiles
+         : f == 30 ? Family{0,   0,  3,  0,   0,  2,  0,  1,  1, 16, -1, 64, 192, -1,  1,  1,  0, -1,  4,  12,  0, -1,  0,  0,  0,  1,  0,  1}     // gather producer, stride 1, wide groups, streamed weights shared by a pair of pixel tiles
                   : Family{-1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1,  -1, -1, -1, -1, -1, -1, -1, -1, -1};
 }
 #define GCONV_FAMILY_FIELDS(X) \
@@ -557,6 +558,9 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 }
                 const uint32_t piece_bytes = (uint32_t)c.CK * (uint32_t)c.boxpx * 4u;
                 const uint32_t part_bytes = (uint32_t)c.pieces * piece_bytes;
+                // pair tiles: a stage (and a raw buffer) holds two pixel tiles, 2 mt and 2 mt + 1, one behind the other
+                const int npt = c.pair ? 2 : 1;
+                const uint32_t mt0 = (uint32_t)npt * mt;
                 for (int ks = 0; ks < kstages; ++ks, ++it) {
                     const uint32_t rs = it % (uint32_t)c.raw_stages, ruse = it / (uint32_t)c.raw_stages;
                     if (ruse > 0 && !mbar_wait_warp(smem_u32(&ctl.raw_empty[rs]), (ruse - 1) & 1u, abort_flag, status, 150 + (int)rs)) { ok = false; break; }
@@ -566,26 +570,26 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     if (c.raw_bulk) {
                         // whole planes of CK consecutive channels are one contiguous run of the input tensor
                         uint32_t live = 0;
-                        for (int pt = 0; pt < c.IPT; ++pt) {
+                        for (int pt = 0; pt < npt * c.IPT; ++pt) {
                             int n, fa;
-                            gath_part(s, c, mt, pt, n, fa);
+                            gath_part(s, c, mt0 + (uint32_t)(pt / c.IPT), pt % c.IPT, n, fa);
                             live += n < s.N ? 1u : 0u;
                         }
                         if (lane == 0) mbar_arrive_expect_tx(rbar, live * part_bytes);
                         __syncwarp();
-                        if (lane < c.IPT) {
+                        if (lane < npt * c.IPT) {
                             int n, fa;
-                            gath_part(s, c, mt, lane, n, fa);
+                            gath_part(s, c, mt0 + (uint32_t)(lane / c.IPT), lane % c.IPT, n, fa);
                             if (n < s.N)
                                 bulk_load_1d(rdst + (uint32_t)lane * part_bytes, x + ((size_t)n * s.C_in + (size_t)chan) * (size_t)HW, part_bytes, rbar);
                         }
                     } else {
-                        if (lane == 0) mbar_arrive_expect_tx(rbar, (uint32_t)c.IPT * part_bytes);   // out-of-range boxes arrive as zeros
+                        if (lane == 0) mbar_arrive_expect_tx(rbar, (uint32_t)(npt * c.IPT) * part_bytes);   // out-of-range boxes arrive as zeros
                         __syncwarp();
-                        if (lane < c.IPT * c.pieces) {
-                            const int pt = lane / c.pieces, pc = lane - pt * c.pieces;
+                        if (lane < npt * c.IPT * c.pieces) {
+                            const int pt = lane / c.pieces, pc = lane - pt * c.pieces;   // pt counts the parts of both tiles
                             int n, fa;
-                            gath_part(s, c, mt, pt, n, fa);
+                            gath_part(s, c, mt0 + (uint32_t)(pt / c.IPT), pt % c.IPT, n, fa);
                             tma_load_3d(rdst + (uint32_t)pt * part_bytes + (uint32_t)pc * piece_bytes, &xmap4, fa + pc * c.boxpx, chan, n, rbar);
                         }
                     }
@@ -792,9 +796,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // zeros.  Then fence.proxy.async, one arrival per copy warp on the stage barrier, one on the raw buffer's.
         // copy warp j builds segment j & 3; in the heavy shape warps 4..7 take the second half of the stage's channels
         const int gw = warp - (c.egroups == 1 ? kEpi2First : kMmaWarp3 + 2);
+        // (pair tiles: warps 4..7 build the stage's second pixel tile instead, all channels)
         const int pw = gw & 3;
-        const int kcount = c.egroups == 2 ? c.CK / 2 : c.CK;            // channels of the stage this warp copies
-        const uint32_t kbase = (uint32_t)(gw >> 2) * (uint32_t)kcount;  // (a multiple of 4: the swizzle term k & 3 is unchanged)
+        const int tp = c.pair ? (gw >> 2) : 0;                          // which tile of the pair
+        const int kcount = (c.egroups == 2 && !c.pair) ? c.CK / 2 : c.CK;   // channels of the stage this warp copies
+        const uint32_t kbase = c.pair ? 0u : (uint32_t)(gw >> 2) * (uint32_t)kcount;  // (a multiple of 4: the swizzle term k & 3 is unchanged)
         const bool g2 = c.soft == 2;
         // lanes take two adjacent pixels (8-byte accesses) when pixel pairs never straddle a row: the two half-warps
         // then take alternate channels
@@ -818,6 +824,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);
             // this warp's segment: image, segment of the image, part of the raw buffer it reads
+            if (c.pair) mt = 2u * mt + (uint32_t)tp;
             int n, i, pt;
             gath_segment(c, mt, pw, n, i, pt);
             int npart, fa;
@@ -833,8 +840,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 // constant offset: the swizzled destination of channel k is base[k & 3] + k * 128 bytes, and the four (two)
                 // bases are computed once per block.  A copy warp is alone with this code on its scheduler, so every
                 // instruction saved shortens the stage's critical path directly.
-                const float* __restrict__ rawp = reinterpret_cast<const float*>(smem + c.raw_off + rs * c.raw_bytes + (uint32_t)pt * part_bytes);
-                float* __restrict__ stg = reinterpret_cast<float*>(smem + (uint32_t)c.b_res * c.bres_stride + (uint32_t)stage * c.stage_bytes);
+                const float* __restrict__ rawp = reinterpret_cast<const float*>(smem + c.raw_off + rs * c.raw_bytes + (uint32_t)(tp * c.IPT + pt) * part_bytes);
+                float* __restrict__ stg = reinterpret_cast<float*>(smem + (uint32_t)c.b_res * c.bres_stride + (uint32_t)stage * c.stage_bytes + (uint32_t)tp * a_bytes);
                 const uint32_t seg_f = seg_bytes >> 2;       // floats per 32-pixel block
                 const uint32_t bpx = (uint32_t)c.boxpx;
                 // (a pointwise layer has the centre tap only: one block, and with stride 2 only the even columns)
@@ -1032,6 +1039,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                             if (c.soft == 2 && !c.pw) {
                                 umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc_e, acc);
                                 umma_tf32_split(d_tmem + (uint32_t)c.Kt, al + 4u * (seg_bytes >> 4), a_hi, bl + (uint32_t)c.Kt, b_hi, idesc_o, acc);
+                                if (c.pair) {                  // same weights, second tile
+                                    umma_tf32_split(d_tmem + (uint32_t)c.Np, al + a_pair16, a_hi, bl, b_hi, idesc_e, acc);
+                                    umma_tf32_split(d_tmem + (uint32_t)(c.Np + c.Kt), al + a_pair16 + 4u * (seg_bytes >> 4), a_hi, bl + (uint32_t)c.Kt, b_hi, idesc_o, acc);
+                                }
                             } else {
                                 umma_tf32_split(d_tmem, al, a_hi, bl, b_hi, idesc, acc);
                                 if (c.pair) umma_tf32_split(d_tmem + (uint32_t)c.Np, al + a_pair16, a_hi, bl, b_hi, idesc, acc);   // same weights, second tile
@@ -1206,11 +1217,18 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        float t = d1[j];
-                        const float up = __shfl_up_sync(0xffffffffu, d0[j], 1u);
-                        const float dn = __shfl_down_sync(0xffffffffu, d2[j], 1u);
-                        if (add_up) t += up;
-                        if (add_dn) t += dn;
+                        float t;
+                        if (c.soft == 2) {                     // columns (centre, left, right): d0 = centre, d1 = left, d2 = right (own lane)
+                            const float up = __shfl_up_sync(0xffffffffu, d1[j], 1u);
+                            t = d0[j] + d2[j];
+                            if (add_up) t += up;
+                        } else {
+                            t = d1[j];
+                            const float up = __shfl_up_sync(0xffffffffu, d0[j], 1u);
+                            const float dn = __shfl_down_sync(0xffffffffu, d2[j], 1u);
+                            if (add_up) t += up;
+                            if (add_dn) t += dn;
+                        }
                         v[kk + j] = t;
                     }
                 }
@@ -1553,6 +1571,7 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     c.Hv = st.H;
     c.Wv = st.W;
     c.CK = c.Cg % 16 == 0 ? 16 : 8;
+    if (heavy && mode == 2) c.CK = 8;            // two pixel tiles of six blocks each share a stage with the streamed weights (pair tiles, below)
     c.chunks = c.Cg / c.CK;
     const int Wo = st.W_out, Ho = st.H_out, HW = st.H * st.W;
     c.rps = 32 / Wo;
@@ -1605,8 +1624,6 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     c.egroups = heavy ? 2 : 1;
     c.threads = heavy ? 32 * (kMmaWarp3 + 2 + 2 * kSoftWarps) : 32 * (kEpi2First + kSoftWarps);
     c.tmem_cols = heavy ? 512 : 256;
-    c.num_tiles = c.groups * c.NT * c.MT;
-    c.div_mt = make_fastdiv((uint32_t)c.MT);
     c.div_spi = make_fastdiv((uint32_t)tpi);
     c.div_w = make_fastdiv((uint32_t)Wo);
     c.div_nt = make_fastdiv((uint32_t)c.NT);
@@ -1619,7 +1636,21 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     c.b_res = 1;
     if (heavy && (b_tile > 144u * 1024u || c.bres_stride + 2u * a_stage + 2u * c.raw_bytes > total || c.MT < 2 * sm_count)) c.b_res = 0;
     c.nt_fast = (!c.b_res && c.NT > 1) ? 1 : 0;
-    c.stage_bytes = (a_stage + (c.b_res ? 0u : (uint32_t)c.nr * (uint32_t)c.Np * (uint32_t)c.CK * 4u) + 1023u) & ~1023u;
+    // Pair tiles: streamed weight blocks cross L2 -> shared memory once per pixel tile, and on wide groups that traffic, not
+    // the tensor core, is the bound.  A stage then holds the operand blocks of TWO pixel tiles and one set of weight blocks;
+    // every weight block feeds two MMAs (two accumulators side by side, one buffer), the eight copy warps build one tile each
+    // per four, and the two epilogue groups drain the two accumulators at the same time.
+    if (heavy && mode == 2) c.b_res = 0;         // (its stages leave no room for a resident bank)
+    if (heavy && !c.b_res && c.MT >= 2 && 2u * a_stage + (uint32_t)c.nr * (uint32_t)c.Np * (uint32_t)c.CK * 4u <= 100u * 1024u) {
+        c.pair = 1;
+        c.MT = (c.MTr + 1) / 2;
+        c.nacc = 1;
+        c.issuers = 1;
+        c.raw_bytes *= 2u;
+    }
+    c.num_tiles = c.groups * c.NT * c.MT;
+    c.div_mt = make_fastdiv((uint32_t)c.MT);
+    c.stage_bytes = ((c.pair ? 2u : 1u) * a_stage + (c.b_res ? 0u : (uint32_t)c.nr * (uint32_t)c.Np * (uint32_t)c.CK * 4u) + 1023u) & ~1023u;
     const uint32_t bank = c.b_res ? c.bres_stride : 0u;
     // the bank, then stages and raw buffers in turn (at most four and four) while they fit; a single stage and a single raw
     // buffer as the last resort
@@ -1633,7 +1664,7 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
         if (c.stages < max_ring && used + c.stage_bytes <= total) { ++c.stages; continue; }
         break;
     }
-    if (heavy && c.stages < 2) return false;
+    if (heavy && (c.stages < 2 || (mode == 2 && !c.pair))) return false;
     c.raw_off = bank + (uint32_t)c.stages * c.stage_bytes;
     c.xchg_off = c.raw_off + (uint32_t)c.raw_stages * c.raw_bytes;
     c.smem_bytes = (size_t)c.xchg_off + 1024;
@@ -2116,7 +2147,7 @@ static cudaError_t igemm_launch(const Shape& s_true, int C2, const float* x_in, 
                                                 igemm_tf32_kernel<14>, igemm_tf32_kernel<15>, igemm_tf32_kernel<16>,
                                                 igemm_tf32_kernel<17>, igemm_tf32_kernel<18>, igemm_tf32_kernel<19>, igemm_tf32_kernel<20>,
                                                 igemm_tf32_kernel<21>, igemm_tf32_kernel<22>, igemm_tf32_kernel<23>,
-                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>, igemm_tf32_kernel<26>, igemm_tf32_kernel<27>, igemm_tf32_kernel<28>, igemm_tf32_kernel<29>};
+                                                igemm_tf32_kernel<24>, igemm_tf32_kernel<25>, igemm_tf32_kernel<26>, igemm_tf32_kernel<27>, igemm_tf32_kernel<28>, igemm_tf32_kernel<29>, igemm_tf32_kernel<30>};
     int fam = 0;
     for (int f = 1; f < kFamilies && fam == 0; ++f)
         if (family_matches(f, s, cfg)) fam = f;

@@ -138,6 +138,11 @@ GATHER_SHAPES = [
     (2, 32, 30, 30, 32, 3, 3, 1, 1, 1, 2), (13, 8, 6, 6, 16, 3, 3, 1, 1, 1, 1), (3, 32, 14, 14, 128, 3, 3, 1, 1, 1, 1),
     (4, 32, 14, 14, 32, 3, 3, 1, 3, 3, 2), (3, 16, 15, 30, 64, 1, 1, 2, 0, 1, 1), (5, 24, 7, 7, 40, 1, 1, 1, 0, 1, 1),
     (2, 192, 15, 30, 1024, 1, 1, 2, 0, 1, 8), (33, 256, 14, 14, 512, 3, 3, 2, 1, 1, 8),
+    # wide groups (one CTA per SM, eight copy warps): a resident bank, streamed banks shared by a pair of pixel tiles with an
+    # odd and an even number of tiles, two filter tiles, stride 2 (8-channel stages), 7x7 planes (two images per tile)
+    (300, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1), (5, 128, 14, 14, 128, 3, 3, 1, 1, 1, 1), (6, 256, 14, 14, 128, 3, 3, 1, 1, 1, 2),
+    (7, 128, 14, 14, 256, 3, 3, 2, 1, 1, 1), (9, 192, 7, 7, 64, 3, 3, 1, 1, 1, 1), (4, 64, 18, 18, 64, 3, 3, 1, 1, 1, 1),
+    (3, 128, 15, 15, 64, 3, 3, 2, 1, 1, 1), (10, 64, 30, 30, 128, 3, 3, 1, 1, 1, 1),
 ]
 
 
