@@ -1555,8 +1555,11 @@ static bool gather_config(IgemmCfg& out, const Shape& st, int sm_count) {
     // Two launch shapes, as for the other producers: narrow (merged) groups run two CTAs per SM with a small resident bank;
     // wide groups (more than 32 channels) run one CTA per SM with 29 warps (eight copy warps behind the two epilogue
     // groups, two per segment), 16-channel stages and the bank resident (up to 144 KB) or streamed with the stages.
-    const bool heavy = c.Cg > 32;
-    if (heavy && (c.pw || c.Cg % 16 != 0 || c.Kt != 64 || st.dilation != 1)) return false;   // (what its two instantiations fix)
+    // (groups of up to 32 channels with 64-filter tiles -- two accumulators do not fit 256 columns -- take the one-CTA shape
+    // too when its instantiations allow; otherwise 32-filter tiles in the two-CTA shape, which gathers every tile twice)
+    const bool heavy_ok = !c.pw && c.Cg % 16 == 0 && c.Kt == 64 && st.dilation == 1;      // (what the one-CTA instantiations fix)
+    const bool heavy = c.Cg > 32 || (2 * c.Np > 256 && heavy_ok);
+    if (heavy && !heavy_ok) return false;
     if (!heavy && !c.pw && 2 * c.Np > 256 && c.Kg % 32 == 0) {           // two accumulators must fit 256 columns: 32-filter tiles
         c.Kt = 32;
         c.NT = c.Kg / 32;
