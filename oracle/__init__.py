@@ -55,6 +55,9 @@ def _load():
             lib.gconv_ref_f64.restype = ctypes.c_int
             lib.gconv_ref_f64.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 11 + [
                 ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
+            lib.gconv_ref_f64_2d.restype = ctypes.c_int
+            lib.gconv_ref_f64_2d.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 14 + [
+                ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
             lib.gconv_ref_out_dim.restype = ctypes.c_int
             lib.gconv_ref_out_dim.argtypes = [ctypes.c_int] * 5
             lib.gconv_ref_max_threads.restype = ctypes.c_int
@@ -71,12 +74,22 @@ def max_threads() -> int:
     return int(_load().gconv_ref_max_threads())
 
 
-def gconv_ref(x: np.ndarray, w: np.ndarray, stride: int = 1, pad: int = 0, dilation: int = 1,
+def _pair(v):
+    """An int stands for both axes; a pair is (rows, columns)."""
+    if isinstance(v, (tuple, list)):
+        if len(v) != 2:
+            raise ValueError("a per-axis parameter is (rows, columns)")
+        return int(v[0]), int(v[1])
+    return int(v), int(v)
+
+
+def gconv_ref(x: np.ndarray, w: np.ndarray, stride=1, pad=0, dilation=1,
               groups: int = 1, threads: int = 1, return_macs: bool = False):
     """Grouped convolution y = gconv(x, w) in fp64.
 
     x: float32 [N, C_in, H, W]; w: float32 [C_out, C_in/groups, KH, KW]; returns float64
-    [N, C_out, H_out, W_out] (and the MAC count of Eq. (2) when ``return_macs``).
+    [N, C_out, H_out, W_out] (and the MAC count of Eq. (2) when ``return_macs``).  stride, pad and dilation are
+    ints (both axes) or (rows, columns) pairs, as Algorithm 1's S_h and S_w.
     """
     x = np.ascontiguousarray(x, dtype=np.float32)
     w = np.ascontiguousarray(w, dtype=np.float32)
@@ -87,14 +100,19 @@ def gconv_ref(x: np.ndarray, w: np.ndarray, stride: int = 1, pad: int = 0, dilat
     if groups < 1 or C_in % groups or C_out % groups or C_in // groups != Cg:
         raise ValueError("channels must split evenly over groups and w.shape[1] == C_in/groups")
     lib = _load()
-    Ho = out_dim(H, KH, stride, pad, dilation)
-    Wo = out_dim(W, KW, stride, pad, dilation)
+    (sh, sw), (ph, pw), (dh, dw) = _pair(stride), _pair(pad), _pair(dilation)
+    Ho = out_dim(H, KH, sh, ph, dh)
+    Wo = out_dim(W, KW, sw, pw, dw)
     if Ho < 1 or Wo < 1:
         raise ValueError("empty output")
     y = np.empty((N, C_out, Ho, Wo), dtype=np.float64)
     macs = ctypes.c_longlong(0)
-    rc = lib.gconv_ref_f64(x.ctypes.data, w.ctypes.data, y.ctypes.data, N, C_in, H, W, C_out, KH, KW,
-                           stride, pad, dilation, groups, int(threads), ctypes.byref(macs))
+    if (sh, ph, dh) == (sw, pw, dw):
+        rc = lib.gconv_ref_f64(x.ctypes.data, w.ctypes.data, y.ctypes.data, N, C_in, H, W, C_out, KH, KW,
+                               sh, ph, dh, groups, int(threads), ctypes.byref(macs))
+    else:
+        rc = lib.gconv_ref_f64_2d(x.ctypes.data, w.ctypes.data, y.ctypes.data, N, C_in, H, W, C_out, KH, KW,
+                                  sh, sw, ph, pw, dh, dw, groups, int(threads), ctypes.byref(macs))
     if rc != 0:
         raise ValueError("gconv_ref_f64 rejected the problem")
     return (y, int(macs.value)) if return_macs else y

@@ -17,6 +17,10 @@
  *   Reads outside [0,H) x [0,W) contribute zero (the paper convolves a padded input).
  *   H_out = floor((H + 2*pad - dilation*(KH-1) - 1) / stride) + 1, likewise W_out.
  *
+ *   Algorithm 1 carries one stride per axis (S_h for rows, S_w for columns); gconv_ref_f64_2d takes stride, padding
+ *   and dilation per axis (row index p*stride_h + r*dilation_h - pad_h, column index q*stride_w + s*dilation_w - pad_w)
+ *   and gconv_ref_f64 is the same sum with both axes given the same values.
+ *
  * Arithmetic: inputs are fp32, every product and the running sum are fp64 (an fp32 x fp32 product
  * is exact in fp64), the result is returned in fp64.  Seven loops: four over the output, three
  * over the reduction.
@@ -41,18 +45,18 @@ int gconv_ref_out_dim(int in, int k, int stride, int pad, int dilation)
 }
 
 /* returns 0 on success, -1 on an invalid problem */
-int gconv_ref_f64(const float *x, const float *w, double *y,
-                  int N, int C_in, int H, int W, int C_out, int KH, int KW,
-                  int stride, int pad, int dilation, int groups,
-                  int threads, long long *macs_out)
+int gconv_ref_f64_2d(const float *x, const float *w, double *y,
+                     int N, int C_in, int H, int W, int C_out, int KH, int KW,
+                     int stride_h, int stride_w, int pad_h, int pad_w, int dilation_h, int dilation_w, int groups,
+                     int threads, long long *macs_out)
 {
     if (N < 1 || C_in < 1 || H < 1 || W < 1 || C_out < 1 || KH < 1 || KW < 1) return -1;
-    if (stride < 1 || pad < 0 || dilation < 1 || groups < 1) return -1;
+    if (stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0 || dilation_h < 1 || dilation_w < 1 || groups < 1) return -1;
     if (C_in % groups != 0 || C_out % groups != 0) return -1;
     const int Cg = C_in / groups;
     const int Kg = C_out / groups;
-    const int H_out = gconv_ref_out_dim(H, KH, stride, pad, dilation);
-    const int W_out = gconv_ref_out_dim(W, KW, stride, pad, dilation);
+    const int H_out = gconv_ref_out_dim(H, KH, stride_h, pad_h, dilation_h);
+    const int W_out = gconv_ref_out_dim(W, KW, stride_w, pad_w, dilation_w);
     if (H_out < 1 || W_out < 1) return -1;
     long long macs = 0;
     if (threads < 1) threads = 1;
@@ -69,8 +73,8 @@ int gconv_ref_f64(const float *x, const float *w, double *y,
                     for (int c = 0; c < Cg; ++c) {
                         for (int r = 0; r < KH; ++r) {
                             for (int s = 0; s < KW; ++s) {
-                                const int h = p * stride + r * dilation - pad;
-                                const int v = q * stride + s * dilation - pad;
+                                const int h = p * stride_h + r * dilation_h - pad_h;
+                                const int v = q * stride_w + s * dilation_w - pad_w;
                                 macs += 1;
                                 if (h >= 0 && h < H && v >= 0 && v < W) {
                                     const size_t xi = (((size_t)n * C_in + (size_t)(g * Cg + c)) * H + h) * W + v;
@@ -87,6 +91,16 @@ int gconv_ref_f64(const float *x, const float *w, double *y,
     }
     if (macs_out) *macs_out = macs;
     return 0;
+}
+
+/* the square case: one stride, padding and dilation for both axes */
+int gconv_ref_f64(const float *x, const float *w, double *y,
+                  int N, int C_in, int H, int W, int C_out, int KH, int KW,
+                  int stride, int pad, int dilation, int groups,
+                  int threads, long long *macs_out)
+{
+    return gconv_ref_f64_2d(x, w, y, N, C_in, H, W, C_out, KH, KW, stride, stride, pad, pad, dilation, dilation, groups,
+                            threads, macs_out);
 }
 
 int gconv_ref_max_threads(void)

@@ -12,13 +12,19 @@ from paper_2006_09791_b200.workloads import Layer
 from golden_io import load_case, load_numbers
 
 GOLDEN_CASES = ["fig3_shape_index_valued.txt", "delta_no_flip.txt", "ones_zero_padding.txt",
-                "stride2_pad1.txt", "dilation2.txt", "two_groups_asymmetric.txt"]
+                "stride2_pad1.txt", "dilation2.txt", "two_groups_asymmetric.txt", "per_axis_stride_pad.txt",
+                "per_axis_dilation.txt"]
+
+
+def _axes(p, key):
+    """A fixture gives one value for both axes (`stride 2`) or one per axis (`stride_h 2 stride_w 3`)."""
+    return p[key] if key in p else (p[key + "_h"], p[key + "_w"])
 
 
 @pytest.mark.parametrize("name", GOLDEN_CASES)
 def test_hand_worked(name):
     x, w, p, y = load_case(name)
-    got, macs = oracle.gconv_ref(x, w, p["stride"], p["pad"], p["dilation"], p["groups"], return_macs=True)
+    got, macs = oracle.gconv_ref(x, w, _axes(p, "stride"), _axes(p, "pad"), _axes(p, "dilation"), p["groups"], return_macs=True)
     assert got.shape == y.shape
     np.testing.assert_array_equal(got, y)  # small integers: exact in fp64
     assert macs == y.size * w.shape[1] * w.shape[2] * w.shape[3]
@@ -95,6 +101,24 @@ def test_matches_torch_conv2d_float64(cfg):
     got = oracle.gconv_ref(x, w, s, p, d, g)
     assert got.shape == tuple(want.shape)
     np.testing.assert_allclose(got, want.numpy(), rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("cfg", [
+    (2, 8, 12, 2, 9, 7, 3, 3, (2, 1), (1, 0), (1, 1)), (1, 6, 6, 3, 11, 8, 3, 2, (1, 3), (2, 1), (2, 1)),
+    (2, 4, 8, 4, 7, 12, 1, 5, (1, 2), (0, 2), (1, 2)), (1, 8, 4, 1, 10, 6, 5, 1, (3, 1), (1, 0), (1, 1))])
+def test_per_axis_parameters_match_torch_conv2d_float64(cfg):
+    """stride, padding and dilation given per axis (S_h, S_w of Algorithm 1): agreement with a library convolution
+    in fp64, and the transposed problem (x and w transposed, every pair swapped) gives the transposed result."""
+    N, C_in, C_out, g, H, W, KH, KW, s, p, d = cfg
+    x = _rand((N, C_in, H, W), 23, 0)
+    w = _rand((C_out, C_in // g, KH, KW), 23, 1)
+    want = torch.nn.functional.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double(), None, s, p, d, g)
+    got, macs = oracle.gconv_ref(x, w, s, p, d, g, return_macs=True)
+    assert got.shape == tuple(want.shape)
+    np.testing.assert_allclose(got, want.numpy(), rtol=0, atol=1e-12)
+    assert macs == got.size * (C_in // g) * KH * KW
+    swapped = oracle.gconv_ref(x.transpose(0, 1, 3, 2), w.transpose(0, 1, 3, 2), s[::-1], p[::-1], d[::-1], g)
+    np.testing.assert_array_equal(swapped, got.transpose(0, 1, 3, 2))
 
 
 def _im2col_matmul(x, w, stride, pad, dilation, groups):
