@@ -80,6 +80,19 @@ enum gconv_variant_id {
 int gconv_desc_create(gconv_desc_t *out, int N, int C_in, int H, int W, int C_out, int KH, int KW,
                       int stride, int pad, int dilation, int groups);
 
+/*
+ * gconv_desc_create_2d -- the same with one stride, padding and dilation per spatial axis: Algorithm 1 of the paper
+ * reads input row oh*S_h + kh and column ow*S_w + kw, i.e. it carries a stride for each axis.
+ *   y[n, g*Kg + k, p, q] = sum_{c, r, s} x[n, g*Cg + c, p*stride_h + r*dilation_h - pad_h, q*stride_w + s*dilation_w - pad_w]
+ *                                        * w[g*Kg + k, c, r, s]
+ *   H_out = floor((H + 2*pad_h - dilation_h*(KH-1) - 1)/stride_h) + 1, W_out likewise with the _w values.
+ * With equal values per axis it is gconv_desc_create.  A problem whose axes differ runs on the FP32 generic variant
+ * (the tensor-core and tiled variants take square parameters only; gconv_variant_supported says so), within the FP32
+ * tolerance.  Host only.  Errors as gconv_desc_create, each condition applied per axis.
+ */
+int gconv_desc_create_2d(gconv_desc_t *out, int N, int C_in, int H, int W, int C_out, int KH, int KW,
+                         int stride_h, int stride_w, int pad_h, int pad_w, int dilation_h, int dilation_w, int groups);
+
 /* Frees the descriptor and its device status block.  NULL is accepted. */
 int gconv_desc_destroy(gconv_desc_t desc);
 

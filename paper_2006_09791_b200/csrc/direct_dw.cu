@@ -398,6 +398,7 @@ dw5_stream_s1_kernel(const Shape s, const DwCfg c, const float* __restrict__ x, 
 }  // namespace
 
 bool dw_supported(const Shape& s) {
+    if (!s.square()) return false;   // one stride, padding and dilation for both axes
     const bool k3 = s.KH == 3 && s.KW == 3 && s.pad == 1, k5 = s.KH == 5 && s.KW == 5 && s.pad == 2;
     if (!((k3 || k5) && s.dilation == 1 && (s.stride == 1 || s.stride == 2))) return false;
     if (!(s.Cg == 1 && s.Kg == 1)) return false;

@@ -1,5 +1,5 @@
 // Variant DIRECT_GENERIC: FP32 FFMA direct grouped convolution, one thread per output element.
-// Handles every shape the descriptor accepts (any kernel size, stride, padding, dilation); it is
+// Handles every shape the descriptor accepts (any kernel size; stride, padding and dilation per axis); it is
 // the safety net of the selector, not a fast path.  Grouped convolution of Section II of the paper,
 // summed in the (c, r, s) order of the convolution stage of Algorithm 1.
 #include "gconv_internal.h"
@@ -53,7 +53,7 @@ generic_forward_kernel(Shape s, const float* __restrict__ x, const uint32_t* __r
                 const int h = p * s.stride + r * s.dilation - s.pad;
                 if (h < 0 || h >= s.H) continue;
                 for (int ss = 0; ss < s.KW; ++ss) {
-                    const int v = q * s.stride + ss * s.dilation - s.pad;
+                    const int v = q * s.stride_w + ss * s.dilation_w - s.pad_w;
                     if (v < 0 || v >= s.W) continue;
                     acc = fmaf(__ldg(xg + ((size_t)c * s.H + h) * s.W + v), __ldg(wk + (c * s.KH + r) * s.KW + ss), acc);
                 }

@@ -195,6 +195,7 @@ FastDiv make_fastdiv(uint32_t d) {
 }
 
 bool rows_supported(const Shape& s) {
+    if (!s.square()) return false;   // one stride, padding and dilation for both axes
     if (!(s.KH == 3 && s.KW == 3 && s.dilation == 1 && (s.stride == 1 || s.stride == 2))) return false;
     if (!(s.Kg == 1 || s.Kg == 2 || s.Kg == 4 || s.Kg == 8)) return false;
     if (s.Cg > 16) return false;

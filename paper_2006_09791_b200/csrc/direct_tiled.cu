@@ -203,6 +203,7 @@ int largest_kt(int Kg) {
 }  // namespace
 
 bool tiled_supported(const Shape& s) {
+    if (!s.square()) return false;   // one stride, padding and dilation for both axes
     if (s.KH == 5 && s.KW == 5) return dw_supported(s);   // 5x5: only the depthwise stream kernel
     return s.KH == 3 && s.KW == 3 && s.dilation == 1 && (s.stride == 1 || s.stride == 2) && s.N <= 65535;
 }

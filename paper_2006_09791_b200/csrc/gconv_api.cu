@@ -79,26 +79,29 @@ IgemmLaunchOpts launch_opts(gconv_desc* d) {
 
 extern "C" {
 
-int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_out, int KH, int KW, int stride,
-                      int pad, int dilation, int groups) {
+int gconv_desc_create_2d(gconv_desc_t* out, int N, int C_in, int H, int W, int C_out, int KH, int KW, int stride_h,
+                         int stride_w, int pad_h, int pad_w, int dilation_h, int dilation_w, int groups) {
     if (out == nullptr) return GCONV_ERR_NULL;
     *out = nullptr;
     if (N < 1 || C_in < 1 || H < 1 || W < 1 || C_out < 1 || KH < 1 || KW < 1) return GCONV_ERR_INVALID_ARG;
-    if (stride < 1 || pad < 0 || dilation < 1 || groups < 1) return GCONV_ERR_INVALID_ARG;
+    if (stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0 || dilation_h < 1 || dilation_w < 1 || groups < 1)
+        return GCONV_ERR_INVALID_ARG;
     if (C_in % groups != 0 || C_out % groups != 0) return GCONV_ERR_INVALID_ARG;
-    const long long span_h = (long long)H + 2LL * pad - (long long)dilation * (KH - 1) - 1;
-    const long long span_w = (long long)W + 2LL * pad - (long long)dilation * (KW - 1) - 1;
+    const long long span_h = (long long)H + 2LL * pad_h - (long long)dilation_h * (KH - 1) - 1;
+    const long long span_w = (long long)W + 2LL * pad_w - (long long)dilation_w * (KW - 1) - 1;
     if (span_h < 0 || span_w < 0) return GCONV_ERR_INVALID_ARG;
     Shape s;
     s.N = N; s.C_in = C_in; s.H = H; s.W = W; s.C_out = C_out; s.KH = KH; s.KW = KW;
-    s.stride = stride; s.pad = pad; s.dilation = dilation; s.groups = groups;
+    s.stride = stride_h; s.pad = pad_h; s.dilation = dilation_h; s.groups = groups;
+    s.stride_w = stride_w; s.pad_w = pad_w; s.dilation_w = dilation_w;
     s.Cg = C_in / groups;
     s.Kg = C_out / groups;
-    s.H_out = (int)(span_h / stride) + 1;
-    s.W_out = (int)(span_w / stride) + 1;
+    s.H_out = (int)(span_h / stride_h) + 1;
+    s.W_out = (int)(span_w / stride_w) + 1;
     const double lim = 1099511627776.0;  // 2^40 elements
     if ((double)N * C_in * H * W > lim || (double)N * C_out * s.H_out * s.W_out > lim ||
-        (double)C_out * s.Cg * KH * KW > 2147483647.0 || (long long)H * W > 2147483647LL || pad > (1 << 20))
+        (double)C_out * s.Cg * KH * KW > 2147483647.0 || (long long)H * W > 2147483647LL || pad_h > (1 << 20) ||
+        pad_w > (1 << 20))
         return GCONV_ERR_INVALID_ARG;
     gconv_desc* d = new (std::nothrow) gconv_desc();
     if (d == nullptr) return GCONV_ERR_INVALID_ARG;
@@ -117,6 +120,11 @@ int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_ou
     d->dbg_skip = -1;
     *out = d;
     return GCONV_OK;
+}
+
+int gconv_desc_create(gconv_desc_t* out, int N, int C_in, int H, int W, int C_out, int KH, int KW, int stride,
+                      int pad, int dilation, int groups) {
+    return gconv_desc_create_2d(out, N, C_in, H, W, C_out, KH, KW, stride, stride, pad, pad, dilation, dilation, groups);
 }
 
 int gconv_desc_destroy(gconv_desc_t d) {

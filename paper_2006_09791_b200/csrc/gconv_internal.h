@@ -9,8 +9,10 @@
 namespace gconv {
 struct Status;
 struct Shape {
-    int N, C_in, H, W, C_out, KH, KW, stride, pad, dilation, groups;
+    int N, C_in, H, W, C_out, KH, KW, stride, pad, dilation, groups;   // stride, pad, dilation: the row axis (S_h of Algorithm 1)
     int Cg, Kg, H_out, W_out;
+    int stride_w, pad_w, dilation_w;                                   // the column axis (S_w); equal to the row values on square problems
+    __host__ __device__ bool square() const { return stride_w == stride && pad_w == pad && dilation_w == dilation; }
 };
 }  // namespace gconv
 

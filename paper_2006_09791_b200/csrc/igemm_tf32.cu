@@ -312,13 +312,13 @@ __host__ __device__ constexpr Family family(int f) {
     //                 rowbox seg nr xchg bres egr s2h lbo str CK  ch  Kt  Np  NT acc iss pad ntf wseg nseg SR f4 tapb fuse ball soft pw
     return f == 1 ? Family{0,   1,  1,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups
          : f == 2 ? Family{0,   1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  0,  0,  0,  0}     // 32-wide planes with halo stages
-         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0,  0,  0}     // row boxes of two segments, narrow groups
+         : f == 3 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 16,  2, 32,  96,  1,  2,  2, -1,  0,  2,   8,  2,  1,  0,  0,  0,  0,  0}     // row boxes of two segments, narrow groups, 16-channel stages
          : f == 4 ? Family{1,   0,  3,  0,   0,  2,  1,  2,  2, 32, -1, 64, 192, -1,  2,  2, -1, -1,  1,   9,  1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, 64-filter tiles, streamed weights
          : f == 5 ? Family{1,   0,  3,  0,   1,  1,  1,  2,  2, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   9, -1,  1,  0,  0,  0,  0,  0}     // stride-2 row tiles, narrow groups
          : f == 6 ? Family{1,   0,  3,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1, -1,  -1, -1,  1,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, streamed weights
          : f == 7 ? Family{1,   0,  3,  0,   1,  2,  0,  1,  1, 32, -1, 64, 192,  1,  2,  2, -1,  0, -1,  -1, -1,  1,  0,  0,  0,  0,  0}     // row boxes, 64-filter tiles, one resident bank
          : f == 8 ? Family{0,   1,  1,  0,   0,  2,  0,  1,  1, 32, -1, 64, 192, -1,  2,  2, -1, -1,  0,   4,  0, -1,  0,  0,  0,  0,  0}     // 16x16 / 8x8 planes, 64-filter tiles, streamed weights
-         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0,  0,  0}     // row boxes of one segment, narrow groups
+         : f == 9 ? Family{1,   0,  3,  0,   1,  1,  0,  1,  1, 16,  2, 32,  96,  1,  2,  2, -1,  0,  1,   6,  1,  1,  0,  0,  0,  0,  0}     // row boxes of one segment, narrow groups, 16-channel stages
          : f == 10 ? Family{0,  1,  3,  0,   1,  1,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2, -1,  0,  4,  12,  0,  0,  1,  0,  0,  0,  0}     // 16x16 / 8x8 planes, narrow groups, tap blocks
          : f == 11 ? Family{0,  1,  3,  0,   1,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  1,   6,  0,  2,  0,  1,  0,  0,  0}     // fused block, 32-wide planes with halo stages
          : f == 12 ? Family{0,  1,  1,  0,   2,  2,  0,  1,  1, 32,  1, 32,  96,  1,  2,  2,  0,  0,  0,   4,  0, -1,  0,  1, -1,  0,  0}     // fused block, 16x16 / 8x8 planes, two resident banks (switching, or one per group)
@@ -1519,6 +1519,7 @@ static int igemm_merge(const Shape& s) {
 }
 
 bool igemm_supported(const Shape& s_any) {
+    if (!s_any.square()) return false;   // one stride, padding and dilation for both axes
     if (s_any.KH == 1 && s_any.KW == 1 && !(s_any.pad == 0 && s_any.dilation == 1)) return false;
     const Shape s = as_3x3(s_any);
     if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.dilation >= 1 && s.pad == s.dilation)) return false;
@@ -1826,6 +1827,16 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     c.fast4 = 0;
     c.nacc = 4 * c.Np <= 512 ? 4 : 2;                 // even, so a buffer always meets the same issuing warp and epilogue group
     c.issuers = c.nacc;                                // MMA-issuing warps: one per accumulator buffer
+    // Row boxes with narrow groups (the two-CTA shape below): stages of 16 channels.  Twice as many stages of half the
+    // size let a tile's first MMAs start when half of its input has arrived and hand shared memory back to the copies
+    // in smaller pieces: 3-7 % on 56x56 and 28x28 planes (256 channels @56x56 N = 32 g = 8: 44.2 -> 42.8 us,
+    // 64 @56x56 N = 64 g = 4: 23.7 -> 22.2 us, 128 @28x28 N = 64 g = 8: 14.3 -> 13.4 us).  Planes 32 pixels wide
+    // (halo stages of whole segments) measured the same either way and keep 32 channels.
+    if (!fuse && !c.pw && c.rowbox && !c.s2h && c.nr == 3 && s.stride == 1 && s.dilation == 1 && c.CK == 32 && c.NT == 1 &&
+        2 * c.Np <= 256 && (uint32_t)vt * (uint32_t)c.Cg * (uint32_t)c.Np * 4u <= 40u * 1024u) {
+        c.CK = 16;
+        c.chunks = c.Cg / 16;
+    }
     // Pair tiles: a filter bank too large to stay resident streams through every CTA's shared memory once per pixel
     // tile, and that traffic (L2 -> shared memory), not the tensor core, bounds the wide layers.  A stage then holds the
     // input of TWO pixel tiles and one set of weight blocks; every weight block feeds two MMAs (one per tile, two

@@ -36,6 +36,7 @@ VARIANT_TOLERANCE = {GCONV_VARIANT_DIRECT_GENERIC: 1e-5, GCONV_VARIANT_DIRECT_TI
 _vp = ctypes.c_void_p
 _SIGNATURES = {
     "gconv_desc_create": (ctypes.c_int, [ctypes.POINTER(_vp)] + [ctypes.c_int] * 11),
+    "gconv_desc_create_2d": (ctypes.c_int, [ctypes.POINTER(_vp)] + [ctypes.c_int] * 14),
     "gconv_desc_destroy": (ctypes.c_int, [_vp]),
     "gconv_out_shape": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]),
     "gconv_macs": (ctypes.c_longlong, [_vp]),
@@ -122,6 +123,14 @@ def gconv_desc_create(N, C_in, H, W, C_out, KH, KW, stride, pad, dilation, group
     h = _vp(0)
     rc = load().gconv_desc_create(ctypes.byref(h), N, C_in, H, W, C_out, KH, KW, stride, pad, dilation, groups)
     _check(rc, "gconv_desc_create")
+    return h.value
+
+
+def gconv_desc_create_2d(N, C_in, H, W, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, dilation_h, dilation_w, groups) -> int:
+    h = _vp(0)
+    rc = load().gconv_desc_create_2d(ctypes.byref(h), N, C_in, H, W, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w,
+                                     dilation_h, dilation_w, groups)
+    _check(rc, "gconv_desc_create_2d")
     return h.value
 
 

@@ -57,6 +57,38 @@ def test_rejects_invalid_descriptors(args):
     assert e.value.status == gconv.GCONV_ERR_INVALID_ARG
 
 
+def test_per_axis_descriptor():
+    """One stride, padding and dilation per axis (S_h and S_w of Algorithm 1): output size by the floor formula per
+    axis; equal axes are the square descriptor; unequal axes leave only the generic FP32 variant."""
+    d = gconv.gconv_desc_create_2d(2, 8, 9, 14, 16, 3, 5, 2, 3, 1, 0, 1, 2, 4)
+    try:
+        assert gconv.gconv_out_shape(d) == ((9 + 2 - 2 - 1) // 2 + 1, (14 + 0 - 2 * 4 - 1) // 3 + 1) == (5, 2)
+        assert gconv.gconv_macs(d) == 2 * 16 * 5 * 2 * 2 * 3 * 5
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_DIRECT_GENERIC
+        assert not gconv.gconv_variant_supported(d, gconv.GCONV_VARIANT_IGEMM_TF32)
+        assert not gconv.gconv_variant_supported(d, gconv.GCONV_VARIANT_DIRECT_TILED)
+        with pytest.raises(gconv.GconvError) as e:
+            gconv.gconv_desc_set_variant(d, gconv.GCONV_VARIANT_IGEMM_TF32)
+        assert e.value.status == gconv.GCONV_ERR_UNSUPPORTED
+    finally:
+        gconv.gconv_desc_destroy(d)
+    for L in config0() + wrn_stack(4, 128)[:3]:
+        a = gconv.gconv_desc_create(*L.desc_args())
+        b = gconv.gconv_desc_create_2d(L.N, L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad,
+                                       L.dilation, L.dilation, L.groups)
+        try:
+            assert gconv.gconv_variant(a) == gconv.gconv_variant(b) and gconv.gconv_packed_bytes(a) == gconv.gconv_packed_bytes(b)
+            assert gconv.gconv_out_shape(a) == gconv.gconv_out_shape(b)
+        finally:
+            gconv.gconv_desc_destroy(a)
+            gconv.gconv_desc_destroy(b)
+    for bad in [(1, 8, 8, 8, 8, 3, 3, 1, 0, 1, 1, 1, 1, 1), (1, 8, 8, 8, 8, 3, 3, 1, 1, 1, -1, 1, 1, 1),
+                (1, 8, 8, 8, 8, 3, 3, 1, 1, 1, 1, 1, 0, 1), (1, 8, 8, 4, 8, 3, 3, 1, 1, 1, 0, 1, 2, 1)]:
+        with pytest.raises(gconv.GconvError) as e:
+            gconv.gconv_desc_create_2d(*bad)
+        assert e.value.status == gconv.GCONV_ERR_INVALID_ARG
+
+
 def test_null_and_variant_errors():
     lib = gconv.load()
     assert lib.gconv_desc_create(None, 1, 8, 8, 8, 8, 3, 3, 1, 1, 1, 1) == gconv.GCONV_ERR_NULL

@@ -46,6 +46,50 @@ def test_hand_worked_cases_on_gpu(name):
             np.testing.assert_allclose(y, y_want, rtol=1e-6, atol=0)
 
 
+PER_AXIS = [  # N, C_in, H, W, C_out, KH, KW, (stride), (pad), (dilation), groups
+    (2, 16, 19, 33, 32, 3, 3, (2, 1), (1, 1), (1, 1), 4), (3, 8, 14, 40, 8, 3, 3, (1, 2), (0, 1), (1, 1), 8),
+    (1, 32, 28, 28, 64, 1, 7, (1, 1), (0, 3), (1, 1), 2), (2, 32, 28, 28, 32, 7, 1, (2, 1), (3, 0), (1, 1), 1),
+    (2, 12, 23, 17, 18, 3, 5, (3, 2), (2, 1), (2, 1), 3), (1, 64, 56, 56, 64, 3, 3, (1, 1), (2, 1), (2, 1), 16),
+    (65, 4, 9, 130, 4, 3, 3, (1, 3), (1, 0), (1, 2), 1)]
+
+
+@pytest.mark.parametrize("cfg", PER_AXIS)
+def test_per_axis_stride_padding_dilation(cfg):
+    """gconv_desc_create_2d (S_h and S_w of Algorithm 1 given separately) against the oracle's per-axis sum, whole
+    tensor, FP32 tolerance; the hand-worked per-axis fixtures exactly."""
+    N, C_in, H, W, C_out, KH, KW, st, pd, dl, g = cfg
+    x, w = synth.make_layer_tensors(N, C_in, H, W, C_out, KH, KW, g, synth.layer_seed(3, N, C_in, H, g))
+    y, used = _run_2d(x, w, st, pd, dl, g)
+    assert used == gconv.GCONV_VARIANT_DIRECT_GENERIC
+    y_ref = oracle.gconv_ref(x, w, st, pd, dl, g, threads=8)
+    assert y.shape == y_ref.shape
+    assert rel_err(y, y_ref) <= gconv.VARIANT_TOLERANCE[used]
+
+
+@pytest.mark.parametrize("name", ["per_axis_stride_pad.txt", "per_axis_dilation.txt"])
+def test_per_axis_hand_worked_cases_on_gpu(name):
+    x, w, p, y_want = load_case(name)
+    y, _ = _run_2d(x, w, (p["stride_h"], p["stride_w"]), (p["pad_h"], p["pad_w"]), (p["dilation_h"], p["dilation_w"]), p["groups"])
+    np.testing.assert_allclose(y, y_want, rtol=1e-6, atol=0)
+
+
+def _run_2d(x_np, w_np, st, pd, dl, g):
+    dev = torch.device("cuda:0")
+    N, C_in, H, W = x_np.shape
+    C_out, _, KH, KW = w_np.shape
+    d = gconv.gconv_desc_create_2d(N, C_in, H, W, C_out, KH, KW, st[0], st[1], pd[0], pd[1], dl[0], dl[1], g)
+    try:
+        Ho, Wo = gconv.gconv_out_shape(d)
+        wp = torch.empty(gconv.gconv_packed_bytes(d) // 4, dtype=torch.float32, device=dev)
+        y = torch.full((N, C_out, Ho, Wo), float("nan"), dtype=torch.float32, device=dev)
+        gconv.gconv_pack_weights(d, torch.from_numpy(w_np).to(dev), wp, None)
+        gconv.gconv_forward(d, torch.from_numpy(x_np).to(dev), wp, y, None)
+        assert gconv.gconv_last_status(d, None) == gconv.GCONV_OK
+        return y.cpu().numpy(), gconv.gconv_variant(d)
+    finally:
+        gconv.gconv_desc_destroy(d)
+
+
 def test_config0_every_variant():
     (L,) = config0()
     ran = 0
