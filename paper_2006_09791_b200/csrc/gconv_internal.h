@@ -92,6 +92,16 @@ struct DwCfg {
     FastDiv div_chunks;
     uint32_t items, blocks;
 };
+// depthwise on small planes (direct_dw_plane.cu): batches of whole planes through shared memory
+struct DwPlaneCfg {
+    int PB, upp;                 // planes per batch, units (one strip of one or two output rows) per plane
+    uint32_t planes, batches, grid, threads, smem_bytes;
+    FastDiv div_upp, div_c;
+};
+bool dw_plane_supported(const Shape& s);
+DwPlaneCfg dw_plane_config(const Shape& s, int sm_count);
+cudaError_t dw_plane_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,
+                             cudaStream_t st);
 bool dw_supported(const Shape& s);
 DwCfg dw_config(const Shape& s, int sm_count);
 cudaError_t dw_forward(const Shape& s, const float* x, const void* packed, float* y, Status* status, int sm_count,

@@ -391,6 +391,25 @@ def test_depthwise_5x5_shapes(cfg):
     check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=5)
 
 
+DW_PLANE_SHAPES = [
+    # N, C, H, W, K, stride: depthwise on planes 7, 14 and 28 pixels wide (batches of whole planes through shared memory):
+    # plane counts that are not a multiple of four or of the batch (a short last batch, or nothing but one), heights that
+    # differ from the width, odd output heights, both filter sizes and strides
+    (3, 5, 7, 7, 3, 1), (1, 3, 7, 7, 5, 1), (2, 6, 9, 14, 5, 2), (5, 7, 20, 28, 3, 2), (9, 33, 14, 14, 3, 1), (4, 9, 5, 7, 3, 2),
+    (3, 4, 28, 28, 5, 2), (2, 64, 13, 14, 5, 1), (1, 2, 30, 28, 5, 1), (7, 11, 28, 28, 5, 1), (2, 50, 7, 7, 5, 2), (6, 96, 14, 14, 5, 2),
+    (1, 1, 7, 7, 3, 1), (13, 20, 3, 14, 3, 1), (2, 130, 27, 28, 3, 2),
+]
+
+
+@pytest.mark.parametrize("cfg", DW_PLANE_SHAPES)
+def test_depthwise_small_planes(cfg):
+    N, C, H, W, K, stride = cfg
+    L = Layer("dwp", N, C, H, W, C, K, K, stride, K // 2, 1, C)
+    err, used = check_layer(L, seed=9)
+    assert used == gconv.GCONV_VARIANT_DIRECT_TILED
+    check_layer(L, gconv.GCONV_VARIANT_DIRECT_GENERIC, seed=9)
+
+
 def test_depthwise_5x5_network_shapes():
     for L in depthwise5x5_layers(N=2):
         check_layer(L)
