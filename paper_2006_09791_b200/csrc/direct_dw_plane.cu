@@ -136,7 +136,8 @@ dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, 
         float* const in = in_buf + buf * in_elems;
         float* const out = out_buf + buf * out_elems;
         if (whole) {
-            if (!bar_wait(smem_addr(&full[buf]), (it >> 1) & 1u)) failed = 1;
+            // one thread polls; the others sleep in the barrier below instead of spending issue slots on the poll loop
+            if (tid == 0 && !bar_wait(smem_addr(&full[buf]), (it >> 1) & 1u)) failed = 1;
             if (__syncthreads_or(failed)) {
                 if (tid == 0) record_status(status, GCONV_ERR_TIMEOUT, 1200 + (int)buf);
                 break;
