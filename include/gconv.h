@@ -62,8 +62,8 @@ enum gconv_variant_id {
     GCONV_VARIANT_DIRECT_TILED = 2,   /* FP32 FFMA, shared-memory halo + register tiles; 3x3, dilation 1, narrow groups;
                                          depthwise 3x3 (pad 1) and 5x5 (pad 2) on a software-pipelined stream kernel */
     GCONV_VARIANT_IGEMM_TF32 = 3      /* TF32 tcgen05 implicit GEMM per (merged) group; 3x3 with pad = dilation or 1x1 with pad 0,
-                                         stride 1 or 2, W <= 128; dilation > 1 only with stride 1 on planes whose (padded)
-                                         rows divide 32 pixels */
+                                         stride 1 or 2 (per axis: gconv_desc_create_2d), W <= 128; dilation > 1 only with
+                                         stride 1 on planes whose (padded) rows divide 32 pixels */
 };
 
 /*
@@ -86,9 +86,11 @@ int gconv_desc_create(gconv_desc_t *out, int N, int C_in, int H, int W, int C_ou
  *   y[n, g*Kg + k, p, q] = sum_{c, r, s} x[n, g*Cg + c, p*stride_h + r*dilation_h - pad_h, q*stride_w + s*dilation_w - pad_w]
  *                                        * w[g*Kg + k, c, r, s]
  *   H_out = floor((H + 2*pad_h - dilation_h*(KH-1) - 1)/stride_h) + 1, W_out likewise with the _w values.
- * With equal values per axis it is gconv_desc_create.  A problem whose axes differ runs on the FP32 generic variant
- * (the tensor-core and tiled variants take square parameters only; gconv_variant_supported says so), within the FP32
- * tolerance.  Host only.  Errors as gconv_desc_create, each condition applied per axis.
+ * With equal values per axis it is gconv_desc_create.  Of the problems whose axes differ the tensor-core variant takes
+ * 3x3 filters with pad 1, dilation 1 and a stride of 2 on one axis only (width a multiple of 4): it computes the stride-1
+ * layer and stores its even rows or columns.  Every other such problem (padding or dilation per axis, other strides)
+ * runs on the FP32 generic variant within the FP32 tolerance; gconv_variant_supported says which applies.  Host only.
+ * Errors as gconv_desc_create, each condition applied per axis.
  */
 int gconv_desc_create_2d(gconv_desc_t *out, int N, int C_in, int H, int W, int C_out, int KH, int KW,
                          int stride_h, int stride_w, int pad_h, int pad_w, int dilation_h, int dilation_w, int groups);

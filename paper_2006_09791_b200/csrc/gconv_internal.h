@@ -145,6 +145,7 @@ struct IgemmCfg {
     int pw;                       // pointwise layer, stride 1: one vertical tap per chunk, one accumulator per filter (N = Kt)
     int soft;                     // gather producer: raw input rows land in a ring by bulk copy, copy warps build the operand stages from
                                   // them (1: stride 1, three vertical-tap blocks; 2: stride 2, even/odd column blocks per tap)
+    int sub_h, sub_w;             // 1: a stride of 2 on that axis, taken as the even rows (columns) of the stride-1 result when it is stored
     int rps, IPT;                 // gather tilings: output rows per 32-lane segment; whole images per tile (1: a tile is part of one image)
     int boxpx, pieces, raw_whole, raw_bulk;   // raw part = `pieces` boxes of boxpx flat pixels x CK channels; parts hold whole planes; one 1-D copy per part
     int raw_stages;               // depth of the raw ring

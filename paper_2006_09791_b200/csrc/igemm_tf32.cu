@@ -1168,9 +1168,9 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             // s.H x s.W is the (possibly padded) plane the kernel computes on; only the first Hv x Wv pixels exist in y
             if (!c.soft) valid = valid && (int)prow < c.Hv && (int)q < c.Wv;
             int fo = c.soft ? g_fo : (int)prow * s.W_out + (int)q;       // position in the output plane
-            if (s.stride == 2 && !c.soft) {              // stride 2 keeps the even rows and columns of the stride-1 result
-                valid = valid && ((prow & 1) == 0) && ((q & 1) == 0);
-                fo = (int)(prow >> 1) * s.W_out + (int)(q >> 1);
+            if (!c.soft && (c.sub_h | c.sub_w)) {        // a stride of 2 keeps the even rows (columns) of the stride-1 result
+                valid = valid && ((prow & (uint32_t)c.sub_h) == 0) && ((q & (uint32_t)c.sub_w) == 0);
+                fo = (int)(prow >> c.sub_h) * s.W_out + (int)(q >> c.sub_w);
             }
             const bool add_up = use_left && lane >= dil;
             const bool add_dn = use_right && lane + dil < 32;
@@ -1345,6 +1345,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constan
         GCONV_FAMILY_FIELDS(GCONV_FIX)
 #undef GCONV_FIX
         if constexpr (fam.stride >= 0) s.stride = fam.stride;
+        if constexpr (fam.stride == 2) c.sub_h = c.sub_w = 1;     // (a stride-1 instantiation also runs the layers with a stride of 2 on one axis)
         s.dilation = 1;
         igemm_tf32_body(xmap, xmap4, s, c, packed, y, status, tag, x);
     }
@@ -1430,6 +1431,9 @@ struct IgemmGeom {
 // divides H*W (14x14 becomes 7x28: no padded copy).
 static Shape as_3x3(const Shape& s) {
     Shape t = s;
+    // One stride per axis (the paper's S_h, S_w) with a stride of 2 on one axis only: every tiling computes the stride-1 layer
+    // and the epilogue stores its even rows or columns (IgemmCfg::sub_h, sub_w), as stride 2 does on planes without row tiles.
+    if (s.stride != s.stride_w) t.stride = t.stride_w = 1;
     if (s.KH == 1 && s.KW == 1) {
         t.KH = 3;
         t.KW = 3;
@@ -1519,7 +1523,13 @@ static int igemm_merge(const Shape& s) {
 }
 
 bool igemm_supported(const Shape& s_any) {
-    if (!s_any.square()) return false;   // one stride, padding and dilation for both axes
+    if (!s_any.square()) {
+        // Per axis only the stride may differ: 3x3, pad 1, dilation 1, strides of 1 and 2, on planes the tiled copies address
+        // (the gather producer and the padded copy build on one stride for both axes).
+        if (s_any.pad_w != s_any.pad || s_any.dilation_w != s_any.dilation || s_any.dilation != 1 || s_any.pad != 1) return false;
+        if (s_any.KH != 3 || s_any.KW != 3 || s_any.W % 4 != 0) return false;
+        if (!((s_any.stride == 1 && s_any.stride_w == 2) || (s_any.stride == 2 && s_any.stride_w == 1))) return false;
+    }
     if (s_any.KH == 1 && s_any.KW == 1 && !(s_any.pad == 0 && s_any.dilation == 1)) return false;
     const Shape s = as_3x3(s_any);
     if (!(s.KH == 3 && s.KW == 3 && (s.stride == 1 || s.stride == 2) && s.dilation >= 1 && s.pad == s.dilation)) return false;
@@ -1701,6 +1711,8 @@ static IgemmCfg igemm_config_c2(const Shape& s_any, int sm_count, int C2) {
     // Pointwise: one vertical tap (a third of the stages and MMAs), one accumulator per filter (N = Kt), filter tiles of
     // up to 128.  Stride 2 computes every pixel and stores the even ones (no stride-2 row tiles: those are built around
     // nine staged rows).
+    c.sub_h = s_any.stride == 2 ? 1 : 0;
+    c.sub_w = s_any.stride_w == 2 ? 1 : 0;
     c.pw = (s_any.KH == 1 && s_any.KW == 1 && C2 == 0) ? 1 : 0;
     const int vt = c.pw ? 1 : 3;
     const bool fuse = C2 > 0;          // fused grouped + pointwise block: heavy shape, streamed or resident grouped weights
@@ -1972,7 +1984,7 @@ IgemmCfg igemm_config(const Shape& s, int sm_count) { return igemm_config_c2(s, 
 
 // ---- fused block: grouped 3x3 followed by a pointwise (1x1, groups = 1) convolution C_out -> C2 ------------------------
 bool igemm_block_supported(const Shape& s, int C2) {
-    if (!igemm_supported(s) || s.KH != 3 || s.stride != 1 || s.dilation != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
+    if (!s.square() || !igemm_supported(s) || s.KH != 3 || s.stride != 1 || s.dilation != 1 || C2 < 16 || C2 > 256 || C2 % 16 != 0) return false;   // C2 is the N of one MMA
     const IgemmCfg c = igemm_config_c2(s, kLayoutSMs, C2);
     if (c.NT != 1 || c.need_xchg || c.padded || c.nacc != 2) return false;
     if (c.d2_col + C2 > c.tmem_cols) return false;

@@ -72,6 +72,14 @@ def test_per_axis_descriptor():
         assert e.value.status == gconv.GCONV_ERR_UNSUPPORTED
     finally:
         gconv.gconv_desc_destroy(d)
+    # strides of 1 and 2 that differ per axis (3x3, pad 1, width a multiple of 4) run on the tensor-core variant
+    d = gconv.gconv_desc_create_2d(4, 64, 28, 28, 64, 3, 3, 2, 1, 1, 1, 1, 1, 4)
+    try:
+        assert gconv.gconv_out_shape(d) == (14, 28)
+        assert gconv.gconv_variant(d) == gconv.GCONV_VARIANT_IGEMM_TF32 and gconv.gconv_workspace_bytes(d) == 0
+        assert not gconv.gconv_block_supported(d, 64)
+    finally:
+        gconv.gconv_desc_destroy(d)
     for L in config0() + wrn_stack(4, 128)[:3]:
         a = gconv.gconv_desc_create(*L.desc_args())
         b = gconv.gconv_desc_create_2d(L.N, L.C_in, L.H, L.W, L.C_out, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad,

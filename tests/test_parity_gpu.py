@@ -66,6 +66,25 @@ def test_per_axis_stride_padding_dilation(cfg):
     assert rel_err(y, y_ref) <= gconv.VARIANT_TOLERANCE[used]
 
 
+PER_AXIS_STRIDE_TC = [  # N, C_in, H, W, C_out, (stride), groups: 3x3, pad 1, a stride of 2 on one axis, planes the tensor-core tilings address
+    (4, 32, 32, 32, 64, (2, 1), 2), (3, 64, 56, 56, 64, (1, 2), 4), (2, 128, 28, 28, 128, (2, 1), 8), (5, 64, 16, 16, 64, (1, 2), 1),
+    (6, 128, 8, 8, 128, (2, 1), 4), (2, 64, 64, 64, 64, (2, 1), 1), (3, 16, 20, 24, 32, (1, 2), 2), (1, 8, 12, 128, 8, (2, 1), 1),
+    (2, 64, 56, 56, 128, (1, 2), 1), (9, 32, 15, 32, 32, (2, 1), 8), (40, 256, 56, 56, 256, (1, 2), 1)]
+
+
+@pytest.mark.parametrize("cfg", PER_AXIS_STRIDE_TC)
+def test_per_axis_stride_on_the_tensor_core_variant(cfg):
+    """S_h != S_w (Algorithm 1) with strides of 1 and 2: the tensor-core variant computes the stride-1 layer and stores its
+    even rows or columns; whole tensor against the per-axis oracle at the TF32 tolerance."""
+    N, C_in, H, W, C_out, st, g = cfg
+    x, w = synth.make_layer_tensors(N, C_in, H, W, C_out, 3, 3, g, synth.layer_seed(4, N, C_in, H, g))
+    y, used = _run_2d(x, w, st, (1, 1), (1, 1), g)
+    assert used == gconv.GCONV_VARIANT_IGEMM_TF32
+    y_ref = oracle.gconv_ref(x, w, st, (1, 1), (1, 1), g, threads=16)
+    assert y.shape == y_ref.shape and np.all(np.isfinite(y))
+    assert rel_err(y, y_ref) <= gconv.VARIANT_TOLERANCE[used]
+
+
 @pytest.mark.parametrize("name", ["per_axis_stride_pad.txt", "per_axis_dilation.txt"])
 def test_per_axis_hand_worked_cases_on_gpu(name):
     x, w, p, y_want = load_case(name)
