@@ -604,6 +604,46 @@ def run_ours(args):
         st = gconv.gconv_last_status(it.desc, stream)
         assert st == 0, gconv.status_string(st)
 
+    # ---- the same step with the five stacks (independent networks) spread over two streams ----------------
+    # Reported beside the headline, not as it: layers of a stack stay in stream order, stacks of different group counts
+    # share no data, so a second stream lets one stack's kernels fill the gaps between the other's dependent launches.
+    side = torch.cuda.Stream(device=dev)
+
+    def step_two_streams():
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        side.wait_event(fork)
+        for k, g in enumerate(wl.WRN_GROUPS):
+            s_k = stream if k % 2 == 0 else side
+            for it in insts:
+                if it.g == g:
+                    gconv.gconv_forward(it.desc, it.x, it.wp, it.y, s_k)
+        join = torch.cuda.Event()
+        join.record(side)
+        stream.wait_event(join)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            step_two_streams()
+        stream.synchronize()
+        side.synchronize()
+        graph2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph2, stream=stream):
+            step_two_streams()
+        graph2.replay()
+        stream.synchronize()
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(args.steps):
+            graph2.replay()
+        e1.record(stream)
+    barrier()
+    ms_two = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    for it in insts:
+        st = gconv.gconv_last_status(it.desc, stream)
+        assert st == 0, gconv.status_string(st)
+
     # ---- end to end through the host-buffer entry point --------------------------------------------
     for _ in range(2):
         step_host()
@@ -758,6 +798,8 @@ def run_ours(args):
                 "clocks": clocks,
                 "e2e": {"value": aggregate_value(step_flops, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                "two_streams": {"ms_per_step": ms_two, "value": aggregate_value(step_flops, world, ms_two), "unit": UNIT,
+                                "how": "the same 90 launches in one CUDA graph, group counts 1, 4, 16 on one stream and 2, 8 on a second"},
                 "gpu_launches": launches_per_step * args.steps,
                 "cpu_baseline": cpu, "layers": rows}
         line.update(extra)
