@@ -87,8 +87,11 @@ struct PlaneGeom {
     static_assert(W_OUT % SW == 0 && (NS & (NS - 1)) == 0, "rows are cut into equal strips");
 };
 
-template <int K, int S, int W>
-__global__ void __launch_bounds__(kPlaneThreads)
+// WHOLE (7x7 planes, stride 1): a thread computes a whole plane -- 49 inputs, the filter and 49 accumulators in
+// registers, every index a compile-time constant, so the instruction stream is the FMAs plus one load and one store
+// per pixel (the strip units above spend half of their instructions on windows, weights and addresses).
+template <int K, int S, int W, bool WHOLE>
+__global__ void __launch_bounds__(WHOLE ? 64 : kPlaneThreads)
 dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, const uint32_t* __restrict__ packed,
                 float* __restrict__ y, Status* status, uint32_t tag) {
     using G = PlaneGeom<K, S, W>;
@@ -147,7 +150,37 @@ dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, 
             for (int i = tid; i < np * HW; i += (int)blockDim.x) in[i] = __ldg(src + i);
             __syncthreads();
         }
-        const int units = np * c.upp;
+        if constexpr (WHOLE) {
+            for (int pl = tid; pl < np; pl += (int)blockDim.x) {
+                uint32_t pq, ch;
+                c.div_c.divmod(plane0 + (uint32_t)pl, pq, ch);
+                const float* __restrict__ wk = wpk + (size_t)ch * (K * K);
+                const float* __restrict__ ip = in + pl * (W * W);
+                float xin[W * W], wr[K * K], acc[W * W];
+#pragma unroll
+                for (int i = 0; i < W * W; ++i) xin[i] = ip[i];
+#pragma unroll
+                for (int i = 0; i < K * K; ++i) wr[i] = __ldg(wk + i);
+#pragma unroll
+                for (int p = 0; p < W; ++p)
+#pragma unroll
+                    for (int q = 0; q < W; ++q) {
+                        float a = 0.f;
+#pragma unroll
+                        for (int r = 0; r < K; ++r)
+#pragma unroll
+                            for (int t = 0; t < K; ++t) {
+                                const int h = p + r - G::PAD, v = q + t - G::PAD;
+                                if (h >= 0 && h < W && v >= 0 && v < W) a = fmaf(xin[h * W + v], wr[r * K + t], a);
+                            }
+                        acc[p * W + q] = a;
+                    }
+                float* __restrict__ op = out + pl * (W * W);
+#pragma unroll
+                for (int i = 0; i < W * W; ++i) op[i] = acc[i];
+            }
+        }
+        const int units = WHOLE ? 0 : np * c.upp;
         for (int u = tid; u < units; u += (int)blockDim.x) {
             uint32_t pl, rem;
             c.div_upp.divmod((uint32_t)u, pl, rem);
@@ -220,10 +253,10 @@ dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, 
     }
 }
 
-template <int K, int S, int W>
+template <int K, int S, int W, bool WHOLE = false>
 cudaError_t launch_plane(const Shape& s, const DwPlaneCfg& c, const float* x, const uint32_t* pk, float* y, Status* status,
                          uint32_t tag, cudaStream_t st) {
-    auto kernel = dw_plane_kernel<K, S, W>;
+    auto kernel = dw_plane_kernel<K, S, W, WHOLE>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -257,7 +290,8 @@ DwPlaneCfg dw_plane_config(const Shape& s, int sm_count) {
     const int per_plane = s.H * s.W + s.H_out * s.W_out;
     const int sw = s.W_out <= 8 ? s.W_out : 7;
     const int rpu = (s.stride == 1 || s.W <= 14) ? 2 : 1;
-    c.upp = ((s.H_out + rpu - 1) / rpu) * (s.W_out / sw);   // a unit is one strip of one (stride 1: two) output rows
+    const bool whole = s.W == 7 && s.H == 7 && s.stride == 1;     // a thread per plane
+    c.upp = whole ? 1 : ((s.H_out + rpu - 1) / rpu) * (s.W_out / sw);   // a unit is one strip of one (stride 1: two) output rows, or a plane
     int pb_max = (50 * 1024) / (per_plane * 8);
     pb_max &= ~3;
     if (pb_max > 64) pb_max = 64;
@@ -265,7 +299,8 @@ DwPlaneCfg dw_plane_config(const Shape& s, int sm_count) {
     double best_eff = -1.0;
     auto threads_for = [&](int pb) {
         const int units = pb * c.upp;
-        return units >= kPlaneThreads ? kPlaneThreads : ((units + 31) / 32) * 32;
+        const int cap = whole ? 64 : kPlaneThreads;
+        return units >= cap ? cap : ((units + 31) / 32) * 32;
     };
     auto ctas_per_sm = [&](int pb) {
         const size_t smem = (size_t)pb * per_plane * 8;
@@ -304,6 +339,7 @@ cudaError_t dw_plane_forward(const Shape& s, const float* x, const void* packed,
     const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed);
 #define GCONV_PLANE_W(K, S) \
     do { \
+        if (s.W == 7 && s.H == 7 && S == 1) return launch_plane<K, 1, 7, true>(s, c, x, pk, y, status, tag, st); \
         if (s.W == 7) return launch_plane<K, S, 7>(s, c, x, pk, y, status, tag, st); \
         if (s.W == 14) return launch_plane<K, S, 14>(s, c, x, pk, y, status, tag, st); \
         return launch_plane<K, S, 28>(s, c, x, pk, y, status, tag, st); \
