@@ -262,7 +262,8 @@ int gconv_last_status(gconv_desc_t desc, void *stream);
 int gconv_last_cuda_error(gconv_desc_t desc);
 
 /* The detail word recorded with the last non-zero device status gconv_last_status returned for this descriptor: for
- * GCONV_ERR_TIMEOUT the wait that gave up (100 + stage: producer waiting for a free stage; 150/160 + buffer: raw ring;
+ * GCONV_ERR_TIMEOUT the wait that gave up (50 + buffer: depthwise plane batches waiting for their bulk copy;
+ * 100 + stage: producer waiting for a free stage; 150/160 + buffer: raw ring;
  * 200 + buffer: accumulator free; 300/800 + stage: MMA waiting for a stage fill; 400 + buffer: epilogue waiting for an
  * accumulator; 500 + buffer: edge exchange; 600/700 + buffer: filter bank; 9xx: fused block), 1000 and up when a drain
  * wait ran out as well; for GCONV_ERR_PACK_MISMATCH the thread block that found it.  Host only; 0 if none. */

@@ -142,7 +142,7 @@ dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, 
             // one thread polls; the others sleep in the barrier below instead of spending issue slots on the poll loop
             if (tid == 0 && !bar_wait(smem_addr(&full[buf]), (it >> 1) & 1u)) failed = 1;
             if (__syncthreads_or(failed)) {
-                if (tid == 0) record_status(status, GCONV_ERR_TIMEOUT, 1200 + (int)buf);
+                if (tid == 0) record_status(status, GCONV_ERR_TIMEOUT, 50 + (int)buf);
                 break;
             }
         } else {
