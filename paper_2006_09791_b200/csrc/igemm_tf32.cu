@@ -898,11 +898,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                         if (c.pw && r != 1) continue;
                         const int h = 2 * p + r - 1;
                         const bool v = lane_ok && h >= 0 && h < s.H;
-                        uint32_t idx = 0;
+                        uint32_t idx = 0, in_piece = 0;
                         if (v) {
                             uint32_t pc, in;
                             c.div_boxpx.divmod((uint32_t)(h * s.W + 2 * q - fa), pc, in);
                             idx = pc * (uint32_t)c.CK * bpx + in;
+                            in_piece = in;
                         }
                         const float* __restrict__ sp = rawp + idx + kbase * bpx;
                         float* __restrict__ dE = stg + (uint32_t)((c.pw ? 0 : r) * 8 + pw) * seg_f + (unit_in >> 2);
@@ -910,7 +911,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 #pragma unroll
                         for (int m = 0; m < 4; ++m) d[m] = dE + kbase * 32u + ((unit_chunk ^ (uint32_t)m) << 3);
                         const uint32_t oblk = 4u * seg_f;    // the odd-column block sits four segments behind the even one
-                        const uint32_t oo = (v && odd_ok) ? 1u : 0u;
+                        // the odd column sits one float behind the even one -- or, on odd widths, where rows start at odd flat
+                        // pixels, at the head of the next piece of the raw part when the even column is a piece's last pixel
+                        const bool has_odd = v && odd_ok;
+                        const uint32_t oo = !has_odd ? 0u : ((!w_even && in_piece + 1u == bpx) ? (uint32_t)c.CK * bpx - in_piece : 1u);
 #pragma unroll
                         for (int k0 = 0; k0 < kcount; k0 += 8) {
                             float e[8], o[8];
@@ -930,7 +934,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                             for (int j = 0; j < 8; ++j) {
                                 float* de = d[(k0 + j) & 3] + (k0 + j) * 32;
                                 de[0] = v ? e[j] : 0.f;
-                                if (!c.pw) de[oblk] = oo ? o[j] : 0.f;
+                                if (!c.pw) de[oblk] = has_odd ? o[j] : 0.f;
                             }
                         }
                     }

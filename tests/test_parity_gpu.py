@@ -138,6 +138,8 @@ ODD_SHAPES = [
     (2, 40, 12, 16, 72, 3, 3, 1, 1, 1, 1), (1, 24, 28, 28, 88, 3, 3, 1, 1, 1, 1), (2, 48, 8, 8, 120, 3, 3, 2, 1, 1, 3),
     (1, 160, 16, 32, 160, 3, 3, 1, 1, 1, 5), (3, 36, 6, 44, 36, 3, 3, 1, 1, 1, 9), (1, 12, 64, 64, 12, 3, 3, 1, 1, 1, 6),
     (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 1), (1, 2, 3, 3, 2, 3, 3, 1, 0, 1, 2), (1, 16, 8, 8, 16, 3, 3, 1, 1, 1, 16),
+    # stride 2 on tall planes of odd width that take the padded copy
+    (2, 32, 48, 15, 32, 3, 3, 2, 1, 1, 2), (1, 128, 57, 29, 128, 3, 3, 2, 1, 1, 4), (2, 16, 70, 27, 32, 3, 3, 2, 1, 1, 1),
     # degenerate planes: one pixel, one row, one column, an output of one pixel
     (2, 8, 1, 1, 8, 3, 3, 1, 1, 1, 2), (1, 8, 1, 9, 16, 3, 3, 1, 1, 1, 1), (1, 16, 2, 2, 16, 3, 3, 2, 1, 1, 4), (3, 8, 1, 7, 8, 3, 3, 1, 1, 1, 8),
     (2, 8, 9, 1, 8, 3, 3, 1, 1, 1, 8), (1, 32, 1, 32, 32, 3, 3, 1, 1, 1, 2), (2, 6, 2, 14, 6, 5, 5, 2, 2, 1, 6), (1, 4, 28, 28, 4, 5, 5, 1, 2, 1, 4),
@@ -209,6 +211,9 @@ GATHER_SHAPES = [
     (300, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1), (5, 128, 14, 14, 128, 3, 3, 1, 1, 1, 1), (6, 256, 14, 14, 128, 3, 3, 1, 1, 1, 2),
     (7, 128, 14, 14, 256, 3, 3, 2, 1, 1, 1), (9, 192, 7, 7, 64, 3, 3, 1, 1, 1, 1), (4, 64, 18, 18, 64, 3, 3, 1, 1, 1, 1),
     (3, 128, 15, 15, 64, 3, 3, 2, 1, 1, 1), (10, 64, 30, 30, 128, 3, 3, 1, 1, 1, 1),
+    # stride 2 on tall planes of odd width: the raw part of a tile comes in several pieces, rows start at odd flat pixels, and an
+    # (even, odd) column pair can straddle two pieces (narrow and wide groups)
+    (2, 64, 64, 31, 64, 3, 3, 2, 1, 1, 1), (3, 32, 64, 31, 64, 3, 3, 2, 1, 1, 1), (3, 512, 64, 31, 512, 3, 3, 2, 1, 1, 4),
 ]
 
 
