@@ -382,8 +382,9 @@ def _seeded_random_shapes(seed, count):
         C, K = g * cg, g * kg
         if C > 512 or K > 512:
             continue
-        H = rng.choice([5, 7, 8, 9, 14, 15, 16, 17, 27, 28, 30, 31, 32, 33, 40, 55, 56, 57, 64])
-        W = rng.choice([5, 6, 7, 8, 12, 13, 14, 15, 16, 20, 24, 28, 29, 30, 31, 32, 36, 40, 48, 52, 56, 60, 64, 96, 128])
+        H = rng.choice([3, 5, 7, 8, 9, 14, 15, 16, 17, 27, 28, 30, 31, 32, 33, 40, 55, 56, 57, 64, 75, 96, 113])
+        W = rng.choice([3, 5, 6, 7, 8, 9, 11, 12, 13, 14, 15, 16, 17, 19, 20, 21, 23, 24, 25, 27, 28, 29, 30, 31, 32, 33, 35, 36, 40, 48, 52, 54,
+                        56, 57, 60, 63, 64, 96, 127, 128])
         stride = rng.choice([1, 1, 1, 2])
         dil = rng.choice([1, 1, 1, 1, 2, 3])
         if H <= 2 * dil or W <= 2 * dil:
@@ -396,7 +397,7 @@ def _seeded_random_shapes(seed, count):
     return out
 
 
-@pytest.mark.parametrize("chunk", range(6))
+@pytest.mark.parametrize("chunk", range(10))
 def test_seeded_random_shapes(chunk):
     for i, cfg in enumerate(_seeded_random_shapes(20260 + chunk, 25)):
         check_layer(Layer("rand%d_%d" % (chunk, i), *cfg), seed=100 * chunk + i)
