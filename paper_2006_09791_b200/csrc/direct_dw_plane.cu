@@ -243,7 +243,8 @@ dw_plane_kernel(const Shape s, const DwPlaneCfg c, const float* __restrict__ x, 
         }
     }
     if (tid == 0) {
-        bulk_store_wait_read<0>();                       // shared memory must outlive the stores that read it
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // every bulk store of this CTA has completed (shared memory must
+                                                                    // outlive the stores that read it; y is whole when the CTA exits)
         // after a wait that ran out a copy may still be in flight into this CTA's shared memory: give it the same limit again
         if (failed) {
             const uint32_t nb = b + gridDim.x;
