@@ -817,6 +817,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         const uint32_t part_bytes = (uint32_t)c.pieces * piece_bytes;
         const int dil = s.dilation;
         uint32_t it = 0;
+        uint32_t rs = 0, ruse = 0;                           // raw ring position of the current fill and its pass over the ring
         int stage = 0;
         uint32_t ph = 0;
         bool ok = true;
@@ -831,8 +832,23 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             gath_part(s, c, mt, pt, npart, fa);
             const int p = i * c.rps + rr;                    // output row of this lane
             const bool lane_ok = n < s.N && i < c.SPI && rr < c.rps && p < s.H_out;
+            // the raw-buffer offsets of this lane's three tap rows do not depend on the channel stage
+            uint32_t tap_idx[3], tap_in[3];
+            bool tap_v[3];
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const int h = g2 ? 2 * p + r - 1 : p + (r - 1) * dil;
+                tap_v[r] = lane_ok && h >= 0 && h < s.H;
+                tap_idx[r] = 0;
+                tap_in[r] = 0;
+                if (tap_v[r]) {
+                    uint32_t pc, in;
+                    c.div_boxpx.divmod((uint32_t)(h * s.W + (g2 ? 2 * q : q) - fa), pc, in);
+                    tap_idx[r] = pc * (uint32_t)c.CK * (uint32_t)c.boxpx + in;
+                    tap_in[r] = in;
+                }
+            }
             for (int ks = 0; ks < kstages; ++ks, ++it) {
-                const uint32_t rs = it % (uint32_t)c.raw_stages, ruse = it / (uint32_t)c.raw_stages;
                 if (!mbar_wait_warp(smem_u32(&ctl.raw_full[rs]), ruse & 1u, abort_flag, status, 160 + (int)rs)) { ok = false; break; }
                 if (it >= (uint32_t)c.stages && !mbar_wait_warp(smem_u32(&ctl.empty[stage]), ph ^ 1, abort_flag, status, 100 + stage)) { ok = false; break; }
                 // Plain shared-memory pointers; a lane with nothing to read loads from the start of its part and stores zeros
@@ -849,14 +865,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 #pragma unroll
                     for (int r = 0; r < 3; ++r) {
                         if (c.pw && r != 1) continue;
-                        const int h = p + (r - 1) * dil;
-                        const bool v = lane_ok && h >= 0 && h < s.H;
-                        uint32_t idx = 0;
-                        if (v) {
-                            uint32_t pc, in;
-                            c.div_boxpx.divmod((uint32_t)(h * s.W + q - fa), pc, in);
-                            idx = pc * (uint32_t)c.CK * bpx + in;
-                        }
+                        const bool v = tap_v[r];
+                        const uint32_t idx = tap_idx[r];
                         float* __restrict__ dp = stg + (uint32_t)((c.pw ? 0 : r) * 4 + pw) * seg_f + (unit_in >> 2);
                         if (pairs) {
                             // half-warp hw takes channels k = 2 j + hw: k & 3 is hw or hw + 2
@@ -896,15 +906,8 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
 #pragma unroll
                     for (int r = 0; r < 3; ++r) {
                         if (c.pw && r != 1) continue;
-                        const int h = 2 * p + r - 1;
-                        const bool v = lane_ok && h >= 0 && h < s.H;
-                        uint32_t idx = 0, in_piece = 0;
-                        if (v) {
-                            uint32_t pc, in;
-                            c.div_boxpx.divmod((uint32_t)(h * s.W + 2 * q - fa), pc, in);
-                            idx = pc * (uint32_t)c.CK * bpx + in;
-                            in_piece = in;
-                        }
+                        const bool v = tap_v[r];
+                        const uint32_t idx = tap_idx[r], in_piece = tap_in[r];
                         const float* __restrict__ sp = rawp + idx + kbase * bpx;
                         float* __restrict__ dE = stg + (uint32_t)((c.pw ? 0 : r) * 8 + pw) * seg_f + (unit_in >> 2);
                         float* __restrict__ d[4];
@@ -946,6 +949,7 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     mbar_arrive(smem_u32(&ctl.raw_empty[rs]));
                 }
                 if (++stage == c.stages) { stage = 0; ph ^= 1; }
+                if (++rs == (uint32_t)c.raw_stages) { rs = 0; ++ruse; }
             }
         }
     } else if (warp == 1 || warp == kMmaWarp2 || warp >= kMmaWarp3) {
