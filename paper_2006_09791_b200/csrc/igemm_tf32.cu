@@ -532,6 +532,11 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
         // One tile's stages: the real copies (arming the stage barriers), or -- pf -- only L2 prefetches of the first
         // pf_limit of them (no barrier).  (Asking L2 for the CTA's next tile while the current one is in flight was
         // measured too: 2 % slower on the stack.)
+        // The dependency wait sits directly in front of the producer's first input copy: tile coordinates, barrier and
+        // buffer addresses of that copy are worked out while the previous kernel is still running, so that what follows
+        // the release of the wait is the copy itself (the producer is one warp walking this code alone: the set-up of a
+        // stage is some hundred instructions, about 600 cycles, in front of every kernel's first load otherwise).
+        bool dep_pending = true;
         auto visit = [&](const int tile, const bool pf, const uint32_t pf_limit, uint32_t& it, int& stage, uint32_t& ph) {
             uint32_t gn, mt;
             tile_coords(c, (uint32_t)tile, gn, mt);      // gn = (group, filter tile) index
@@ -567,6 +572,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                     const uint32_t rbar = smem_u32(&ctl.raw_full[rs]);
                     const uint32_t rdst = smem_base + c.raw_off + rs * c.raw_bytes;
                     const int chan = g * c.Cg + ks * c.CK;
+                    if (dep_pending) {
+                        asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
+                        dep_pending = false;
+                    }
                     if (c.raw_bulk) {
                         // whole planes of CK consecutive channels are one contiguous run of the input tensor
                         uint32_t live = 0;
@@ -651,6 +660,10 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const bool skip_fill = !pf && (int)it == c.dbg_skip && blockIdx.x == 0;
                 const int lo = tile_f0 + (r - 1) * rstep - c.wseg * 32;
                 const bool box = c.rowbox || c.fast4 == 2 || (c.fast4 == 1 && lo >= 0 && lo + c.nseg * 32 <= HW);
+                if (!pf && dep_pending) {
+                    asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
+                    dep_pending = false;
+                }
                 if (skip_fill) {
                     // nothing
                 } else if (lane == 0 && pf) {
@@ -720,7 +733,6 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             for (int tile = tile_first; tile < tile_end && it < kPrefetchUses; tile = tile_next(tile)) visit(tile, true, kPrefetchUses, it, stage, ph);
             run_epilogue = true;
         } else {
-            asm volatile("griddepcontrol.wait;" ::: "memory");   // the input may be the previous kernel's output
             for (int tile = tile_first; tile < tile_end && ok; tile = tile_next(tile)) visit(tile, false, 0u, it, stage, ph);
         }
         if (producer && !ok && lane == 0) {
