@@ -1045,12 +1045,13 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)c.Np;
                 uint32_t acc = 0;
                 for (int ks = 0; ks < kstages; ++ks) {
-                    if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 300 + stage)) { ok = false; break; }
-                    tc_fence_after();
+                    // (the descriptors of the stage are worked out before the wait: what follows the arrival of the data is the MMAs)
                     const uint32_t a16 = (stage_base + (uint32_t)stage * c.stage_bytes) >> 4;
                     // weights of this stage: (chunk, tap) blocks of the resident bank, or the blocks staged behind A
                     const uint32_t b16 = c.b_res ? (bres_addr >> 4) + (uint32_t)(c.nr == 3 ? ks * 3 : ks) * blk16 : a16 + b_in_stage16;
                     uint32_t alo = a_lo0 + a16, blo = b_lo0 + b16;
+                    if (!mbar_wait(smem_u32(&ctl.full[stage]), ph, abort_flag, status, 300 + stage)) { ok = false; break; }
+                    tc_fence_after();
                     // tap r of a halo stage is the view that starts r rows (wseg segments per row) further in
                     for (int rr = 0; rr < c.nr; ++rr, alo += view16, blo += blk16) {
                         uint32_t al = alo, bl = blo;
@@ -1194,11 +1195,12 @@ igemm_tf32_body(const CUtensorMap& xmap, const CUtensorMap& xmap4, const Shape& 
             }
             const bool add_up = use_left && lane >= dil;
             const bool add_dn = use_right && lane + dil < 32;
-            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), bph, abort_flag, status, 400 + buf)) break;
-            tc_fence_after();
+            // (addresses first, then the wait for the accumulator: what follows the MMAs' completion is the reads and the stores)
             const uint32_t t0 = tmem_base + (c.pair ? egroup : buf) * (uint32_t)c.Np + ((uint32_t)(wq * 32) << 16);
             // output channel of filter 0 of this tile: gn*Kt == g*Kg_eff + nt*Kt
             float* yk = y + ((size_t)n * s.C_out + (size_t)gn * Kt + (size_t)kbeg) * OHW + fo;
+            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), bph, abort_flag, status, 400 + buf)) break;
+            tc_fence_after();
             // fused block: this lane's slot in the A2 operand (32-pixel block wq, 128-byte row per channel, 32-byte
             // chunks swizzled by the channel index), once the pointwise MMAs of the buffer's previous use are done
             uint8_t* a2p = smem + c.a2_off + (size_t)egroup * 4u * (size_t)Kt * 128u + (size_t)wq * (size_t)Kt * 128u + (size_t)(lane & 7) * 4u;
